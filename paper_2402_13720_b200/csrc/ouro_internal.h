@@ -1,0 +1,133 @@
+// Internal declarations shared by the translation units of libouro (not part of the public ABI).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include <string>
+#include <vector>
+
+#include "ouro.h"
+
+typedef unsigned long long u64;
+
+// Device-resident scalars of one decoding stream.
+struct DevState {
+  int32_t pending;   // last accepted token; its K/V is not cached yet (block row 0 of the next step)
+  int32_t n_seq;     // tokens of the text recorded in seq_dev (== target cache length + 1)
+  int32_t n_cand;    // candidates found by the last lookup (K' <= K)
+  int32_t n_rows;    // rows of the last assembled target block
+  int32_t A;         // accurate draft prefix of the last verification (Eq. 3)
+  int32_t chosen;    // chosen candidate or -1
+  int32_t m;         // matched suffix tokens of the chosen candidate (hat-A - 1, Eq. 9)
+  int32_t n_acc;     // tokens accepted by the last verification
+  int32_t accepted[OURO_MAX_GAMMA + OURO_MAX_BETA];
+  int32_t status;    // sticky device-side error word (0 = fine)
+  int32_t pad;
+  u64 clock;         // phrase-pool stamp counter
+};
+
+// Per-row description of a query block.  Row r attends, in this order, cache slots [0, lin_end[r])
+// and then slots [seg_start[r], seg_start[r] + seg_len[r]): the "virtual position" p of a key maps
+// to slot p (p < lin_end) or seg_start + p - lin_end.  A trunk row has seg_len == 0; the suffix row
+// (j, i) of Eq. 8 has lin_end = L + gamma + 1 and its own candidate's first i suffix slots.
+struct BlockDev {
+  int32_t *tok, *pos, *group, *lin_end, *seg_start, *seg_len;
+  u64 *mask;  // [rows][2] visibility inside the block, for inspection only (kernels use the ranges)
+};
+
+struct PoolDev {
+  int32_t *key;   // [sets*ways], -1 = free
+  int32_t *suf;   // [sets*ways, S]
+  u64 *stamp;     // [sets*ways]
+  int32_t sets, ways, S;
+};
+
+struct ModelRt {
+  bool present = false;
+  ouro_model_desc d{};
+  const void *embed = nullptr, *final_norm = nullptr, *lm_head = nullptr;
+  std::vector<const void *> attn_norm, wq, wk, wv, wo, ffn_norm, w_gate, w_up, w_down;
+  void *k_cache = nullptr, *v_cache = nullptr;
+  float *rope_cos = nullptr, *rope_sin = nullptr;  // [max_seq, head_dim/2], filled at create
+  BlockDev blk{};
+  int32_t L = 0;        // cache length (host mirror)
+  int32_t blk_rows = 0; // rows of the current block (0 = none assembled)
+  int32_t blk_L = -1;   // cache length the block was assembled for
+  bool blk_is_candidate = false;
+};
+
+struct Activations {  // sized for OURO_MAX_ROWS rows of the larger model
+  float *x;        // residual stream [rows, d_model]
+  void *xn;        // normed activations [rows, d_model], model dtype
+  float *qkv;      // [rows, d_q + 2 d_kv]
+  void *q;         // rotated queries [rows, d_q], model dtype
+  void *att;       // attention output [rows, d_q], model dtype
+  void *act;       // SwiGLU output [rows, d_ffn], model dtype
+  float *logits;   // [rows, vocab]
+  int32_t *argmax; // [rows]
+  float *scratch;  // split-K partial sums / split-KV partial softmax states
+  size_t scratch_bytes;
+};
+
+struct ouro_ctx {
+  ModelRt m[2];
+  ouro_params p{};
+  cudaStream_t stream = nullptr;
+  Activations a{};
+  DevState *st = nullptr;
+  int32_t *seq_dev = nullptr;     // [max_seq of target]
+  int32_t *cand_suffix = nullptr; // [K, S]
+  int32_t *cand_count = nullptr;  // [1]
+  int32_t *draft_dev = nullptr;   // [gamma]
+  int32_t *stage_dev = nullptr;   // [OURO_MAX_ROWS] staging for token uploads
+  PoolDev pool{};
+  // host side
+  std::vector<int32_t> seq;       // the text: prompt + accepted tokens (last one pending)
+  int32_t *pin = nullptr;         // pinned host staging (PIN_INTS ints)
+  ouro_drafter_fn drafter = nullptr;
+  void *drafter_user = nullptr;
+  int32_t step = 0;
+  std::string err;
+  cudaEvent_t ev[6] = {nullptr, nullptr, nullptr, nullptr, nullptr, nullptr};
+};
+enum { PIN_INTS = 1024 };
+
+// ---- kernel launchers (kernels_block.cu) ---------------------------------------------------------
+void launch_pool_clear(const PoolDev &P, DevState *st, cudaStream_t s);
+void launch_pool_lookup(const PoolDev &P, const int32_t *key_dev, int key_index, int K, int32_t *suffix, int32_t *count,
+                        cudaStream_t s);
+void launch_pool_update(const PoolDev &P, DevState *st, const int32_t *ngrams, int n, int beta, cudaStream_t s);
+void launch_assemble_candidates(const BlockDev &b, DevState *st, const int32_t *draft, const int32_t *suffix,
+                                const int32_t *count, int L, int gamma, int S, int K, cudaStream_t s);
+void launch_assemble_causal(const BlockDev &b, const int32_t *tokens, int n, int L, cudaStream_t s);
+void launch_accept(const BlockDev &b, DevState *st, const int32_t *o, int32_t *seq_dev, int gamma, int S,
+                   cudaStream_t s);
+void launch_compact(const ouro_model_desc &d, void *k_cache, void *v_cache, const DevState *st, int L, int gamma,
+                    int S, cudaStream_t s);
+void launch_harvest(const BlockDev &b, DevState *st, const PoolDev &P, const int32_t *o, const int32_t *seq_dev,
+                    int gamma, int S, unsigned flags, cudaStream_t s);
+void launch_argmax(const float *logits, int rows, int vocab, int32_t *out, cudaStream_t s);
+void launch_pick_token(const int32_t *src, int index, int32_t *dst, cudaStream_t s);
+void launch_set_state(DevState *st, int32_t *seq_dev, int n_seq, int pending, cudaStream_t s);
+
+// ---- kernel launchers (kernels_layer.cu) ---------------------------------------------------------
+struct GemmSegs {  // up to three weight matrices [n_i, K] stacked along the output dimension
+  const void *w[3];
+  int n[3];
+  int count;
+};
+enum { EPI_STORE = 0, EPI_RESIDUAL = 1 };
+void launch_rope_table(float *cos_t, float *sin_t, int max_seq, int head_dim, float theta, cudaStream_t s);
+void launch_embed(int dtype, const void *E, const int32_t *tok, int rows, int d, float *x, cudaStream_t s);
+void launch_rmsnorm(int dtype, const float *x, const void *g, int rows, int d, float eps, void *out, cudaStream_t s);
+void launch_gemm_simple(int dtype, const void *X, const GemmSegs &W, int rows, int K, float *Y, int ldy, int epi,
+                        cudaStream_t s);
+void launch_gemm_swiglu_simple(int dtype, const void *X, const void *Wg, const void *Wu, int rows, int K, int F,
+                               void *act, cudaStream_t s);
+void launch_rope_append(const ouro_model_desc &d, const float *qkv, const int32_t *pos, const float *cos_t,
+                        const float *sin_t, int rows, int L, int layer, void *q, void *k_cache, void *v_cache,
+                        cudaStream_t s);
+void launch_attention_simple(const ouro_model_desc &d, const void *q, const void *k_cache, const void *v_cache,
+                             const BlockDev &b, int rows, int layer, void *out, cudaStream_t s);
