@@ -118,16 +118,18 @@ __global__ void pool_clear_kernel(PoolDev P, DevState *st) {
   if (i == 0) st->clock = 0;
 }
 
-__global__ void pool_lookup_kernel(PoolDev P, const int32_t *key_dev, int key_index, int K, int32_t *suffix,
-                                   int32_t *count) {
-  int n = key_dev[key_index] < 0 ? 0 : pool_lookup(P, key_dev[key_index], K, suffix);
+__global__ void pool_lookup_kernel(PoolDev P, const int32_t *key_dev, int key_index, int32_t key_value, int K,
+                                   int32_t *suffix, int32_t *count) {
+  int32_t key = key_dev ? key_dev[key_index] : key_value;
+  int n = (key < 0 || P.S == 0) ? 0 : pool_lookup(P, key, K, suffix);
   if (threadIdx.x == 0) *count = n;
 }
 
-__global__ void pool_update_kernel(PoolDev P, DevState *st, const int32_t *ngrams, int n, int beta) {
+// n beta-grams, the g-th starting at ngrams + g*stride (stride 1 = sliding windows over a text).
+__global__ void pool_update_kernel(PoolDev P, DevState *st, const int32_t *ngrams, int n, int beta, int stride) {
   int32_t ph[OURO_MAX_BETA];
   for (int g = 0; g < n; ++g) {
-    for (int i = 0; i < beta; ++i) ph[i] = ngrams[(size_t)g * beta + i];
+    for (int i = 0; i < beta; ++i) ph[i] = ngrams[(size_t)g * stride + i];
     pool_insert(P, st, ph);
   }
 }
@@ -136,12 +138,13 @@ void launch_pool_clear(const PoolDev &P, DevState *st, cudaStream_t s) {
   int n = P.sets * P.ways;
   pool_clear_kernel<<<(n + 255) / 256, 256, 0, s>>>(P, st);
 }
-void launch_pool_lookup(const PoolDev &P, const int32_t *key_dev, int key_index, int K, int32_t *suffix, int32_t *count,
-                        cudaStream_t s) {
-  pool_lookup_kernel<<<1, 32, 0, s>>>(P, key_dev, key_index, K, suffix, count);
+void launch_pool_lookup(const PoolDev &P, const int32_t *key_dev, int key_index, int32_t key_value, int K,
+                        int32_t *suffix, int32_t *count, cudaStream_t s) {
+  pool_lookup_kernel<<<1, 32, 0, s>>>(P, key_dev, key_index, key_value, K, suffix, count);
 }
-void launch_pool_update(const PoolDev &P, DevState *st, const int32_t *ngrams, int n, int beta, cudaStream_t s) {
-  pool_update_kernel<<<1, 32, 0, s>>>(P, st, ngrams, n, beta);
+void launch_pool_update(const PoolDev &P, DevState *st, const int32_t *ngrams, int n, int beta, int stride,
+                        cudaStream_t s) {
+  if (n > 0) pool_update_kernel<<<1, 32, 0, s>>>(P, st, ngrams, n, beta, stride);
 }
 
 // --------------------------------------------------------------------------- candidate packing
@@ -373,16 +376,27 @@ void launch_argmax(const float *logits, int rows, int vocab, int32_t *out, cudaS
   argmax_kernel<<<rows, 256, 0, s>>>(logits, vocab, out);
 }
 
+// Plain greedy decoding: the row-0 output becomes the next pending token and joins the text.
+__global__ void vanilla_accept_kernel(DevState *st, const int32_t *o, int32_t *seq_dev) {
+  st->pending = o[0];
+  seq_dev[st->n_seq] = o[0];
+  st->n_seq += 1;
+}
+void launch_vanilla_accept(DevState *st, const int32_t *o, int32_t *seq_dev, cudaStream_t s) {
+  vanilla_accept_kernel<<<1, 1, 0, s>>>(st, o, seq_dev);
+}
+
 __global__ void pick_token_kernel(const int32_t *src, int index, int32_t *dst) { *dst = src[index]; }
 void launch_pick_token(const int32_t *src, int index, int32_t *dst, cudaStream_t s) {
   pick_token_kernel<<<1, 1, 0, s>>>(src, index, dst);
 }
 
-// n_seq - 1 cached text positions recorded as token 0, then the pending token.
-__global__ void set_state_kernel(DevState *st, int32_t *seq_dev, int n_seq, int pending) {
-  for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < n_seq; i += gridDim.x * blockDim.x)
-    seq_dev[i] = i == n_seq - 1 ? pending : 0;
+// Text of n_seq tokens ending in the pending token; with fill, the earlier positions are recorded as 0.
+__global__ void set_state_kernel(DevState *st, int32_t *seq_dev, int n_seq, int pending, int fill) {
+  if (fill)
+    for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < n_seq - 1; i += gridDim.x * blockDim.x) seq_dev[i] = 0;
   if (blockIdx.x == 0 && threadIdx.x == 0) {
+    seq_dev[n_seq - 1] = pending;
     st->pending = pending;
     st->n_seq = n_seq;
     st->n_cand = 0;
@@ -390,6 +404,6 @@ __global__ void set_state_kernel(DevState *st, int32_t *seq_dev, int n_seq, int 
     st->status = 0;
   }
 }
-void launch_set_state(DevState *st, int32_t *seq_dev, int n_seq, int pending, cudaStream_t s) {
-  set_state_kernel<<<8, 256, 0, s>>>(st, seq_dev, n_seq, pending);
+void launch_set_state(DevState *st, int32_t *seq_dev, int n_seq, int pending, int fill, cudaStream_t s) {
+  set_state_kernel<<<8, 256, 0, s>>>(st, seq_dev, n_seq, pending, fill);
 }

@@ -96,9 +96,11 @@ enum { PIN_INTS = 1024 };
 
 // ---- kernel launchers (kernels_block.cu) ---------------------------------------------------------
 void launch_pool_clear(const PoolDev &P, DevState *st, cudaStream_t s);
-void launch_pool_lookup(const PoolDev &P, const int32_t *key_dev, int key_index, int K, int32_t *suffix, int32_t *count,
+void launch_pool_lookup(const PoolDev &P, const int32_t *key_dev, int key_index, int32_t key_value, int K,
+                        int32_t *suffix, int32_t *count, cudaStream_t s);
+void launch_pool_update(const PoolDev &P, DevState *st, const int32_t *ngrams, int n, int beta, int stride,
                         cudaStream_t s);
-void launch_pool_update(const PoolDev &P, DevState *st, const int32_t *ngrams, int n, int beta, cudaStream_t s);
+void launch_vanilla_accept(DevState *st, const int32_t *o, int32_t *seq_dev, cudaStream_t s);
 void launch_assemble_candidates(const BlockDev &b, DevState *st, const int32_t *draft, const int32_t *suffix,
                                 const int32_t *count, int L, int gamma, int S, int K, cudaStream_t s);
 void launch_assemble_causal(const BlockDev &b, const int32_t *tokens, int n, int L, cudaStream_t s);
@@ -110,7 +112,7 @@ void launch_harvest(const BlockDev &b, DevState *st, const PoolDev &P, const int
                     int gamma, int S, unsigned flags, cudaStream_t s);
 void launch_argmax(const float *logits, int rows, int vocab, int32_t *out, cudaStream_t s);
 void launch_pick_token(const int32_t *src, int index, int32_t *dst, cudaStream_t s);
-void launch_set_state(DevState *st, int32_t *seq_dev, int n_seq, int pending, cudaStream_t s);
+void launch_set_state(DevState *st, int32_t *seq_dev, int n_seq, int pending, int fill, cudaStream_t s);
 
 // ---- kernel launchers (kernels_layer.cu) ---------------------------------------------------------
 struct GemmSegs {  // up to three weight matrices [n_i, K] stacked along the output dimension
