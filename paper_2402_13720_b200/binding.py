@@ -155,7 +155,7 @@ class Engine:
             raise RuntimeError("a CUDA device is required: this library has no CPU path")
         self.L = lib()
         self.device = torch.device(device)
-        self.target, self.draft, self.params = target, draft, params
+        self.target_desc, self.draft_desc, self.params = target, draft, params
         self.tm = _ModelMem(target, target_w, self.device)
         self.dm = _ModelMem(draft, draft_w, self.device) if draft is not None else None
         self._td, self._pd = desc_c(target), params_c(params)
