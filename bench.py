@@ -1,0 +1,325 @@
+"""Benchmark of the Ouroboros verification step on B200.
+
+A step is one pass of the whole hot path over one synthetic batch: phrase lookup, candidate packing, one
+target forward under the candidate mask (embedding, decoder layers, LM head, argmax), greedy acceptance,
+KV compaction and phrase harvest.  Workload: one 7B-shaped decoder layer (d 4096, 32 heads, FFN 11008,
+vocabulary 32000, bf16) on a 4096-token KV cache with a 37-row query block (1 + 4 draft tokens + 4 phrases
+x 8 tokens).  The metric is the verify-step HBM throughput: algorithmic bytes of the step / step time.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--cache-len L]
+
+N > 1 runs N independent replicas (one process per GPU under torchrun); the decoding stream of one query is
+strictly sequential, so there is no data-path collective.  `--impl reference` times the CPU oracle.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import sys
+import threading
+import time
+
+import numpy as np
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2402_13720_b200 import synth  # noqa: E402
+
+METRIC, UNIT = "verify_step_hbm_throughput", "GB/s"
+SEED = 0
+PENDING = 17
+PROF_CLASSES = ("qkv", "attention", "wo", "gateup", "down", "head")
+
+
+# ------------------------------------------------------------------------------ workload
+
+def algorithmic_bytes(m: synth.ModelDesc, B: int, L: int) -> dict:
+    """Bytes one verification step must move: every weight once, the visible KV cache once, the block's K/V
+    written once, B embedding rows; activations (a few hundred KB, L2 resident) are not counted."""
+    e = 2 if m.dtype == "bf16" else 4
+    layer_w = m.layer_weight_elems() * e + 2 * m.d_model * e
+    kv_read = 2 * L * m.d_kv * e
+    kv_write = 2 * B * m.d_kv * e
+    per_class = {
+        "qkv": (m.d_q + 2 * m.d_kv) * m.d_model * e,
+        "attention": kv_read + 2 * B * m.d_kv * e,
+        "wo": m.d_model * m.d_q * e,
+        "gateup": 2 * m.d_ffn * m.d_model * e,
+        "down": m.d_ffn * m.d_model * e,
+        "head": m.vocab * m.d_model * e,
+    }
+    total = m.n_layers * (layer_w + kv_read + kv_write) + m.vocab * m.d_model * e + m.d_model * e + B * m.d_model * e
+    return dict(total=total, per_class=per_class, layers=m.n_layers)
+
+
+def block_inputs(m: synth.ModelDesc, P: synth.DecodeParams):
+    """Seeded draft tokens and K phrases that start with the draft's last token."""
+    draft = np.array([synth.hash_u64(SEED, 70, i) % m.vocab for i in range(P.gamma)], dtype=np.int32)
+    grams = np.array([[draft[-1]] + [synth.hash_u64(SEED, 71, j * 64 + i) % m.vocab for i in range(P.S)]
+                      for j in range(P.K)], dtype=np.int32)
+    return draft, grams
+
+
+class GpuWorkload:
+    def __init__(self, device, cache_len):
+        from paper_2402_13720_b200 import binding, build
+        build.build()
+        self.m, _, self.P, _ = synth.config("C2")
+        if cache_len + self.P.block_max + 1 > self.m.max_seq:
+            raise SystemExit("cache length does not fit the configuration's max_seq")
+        self.L = cache_len
+        self.w = synth.model_weights(self.m, SEED, device=device)
+        self.eng = binding.Engine(self.m, self.w, self.P, device=device)
+        k, v = synth.kv_fill(self.m, SEED + 1, cache_len, device=device)
+        self.eng.tm.k_cache.copy_(k)
+        self.eng.tm.v_cache.copy_(v)
+        self.draft, self.grams = block_inputs(self.m, self.P)
+        self.eng.phrase_update(self.grams)
+        self.eng.draft_tokens.copy_(torch.as_tensor(self.draft, device=device))
+        self.draft_pinned = torch.as_tensor(self.draft).pin_memory()
+        self.B = self.P.block_max
+        self.bytes = algorithmic_bytes(self.m, self.B, self.L)
+
+    def step(self, host_inputs=False):
+        e = self.eng
+        e.set_state(self.L, PENDING)
+        if host_inputs:                               # end-to-end: the step's inputs start in pinned host memory
+            e.draft_tokens.copy_(self.draft_pinned, non_blocking=True)
+        e.assemble_candidates()
+        e.verify_forward()
+        return e.accept_and_compact()                 # returns host values: a device->host read per step
+
+    def check(self):
+        n, chosen, A, acc = self.step()
+        assert self.eng.block_get()[0].shape[0] == self.B, "the pool no longer yields K candidates"
+        assert 1 <= n <= self.P.gamma + self.P.beta
+        return n
+
+
+# -------------------------------------------------------------------------------- clocks
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons through NVML while the timed region runs."""
+
+    def __init__(self, index):
+        self.samples, self.reasons, self.max_mhz, self._stop = [], set(), None, threading.Event()
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+        except Exception:
+            self.nv = None
+        self.t = threading.Thread(target=self._run, daemon=True)
+
+    def _run(self):
+        nv = self.nv
+        names = {"hw_slowdown": 0x8, "sw_power_cap": 0x4, "hw_thermal_slowdown": 0x40, "sw_thermal_slowdown": 0x20,
+                 "hw_power_brake": 0x80}
+        while not self._stop.is_set():
+            try:
+                self.samples.append(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
+                r = nv.nvmlDeviceGetCurrentClocksEventReasons(self.h) if hasattr(nv, "nvmlDeviceGetCurrentClocksEventReasons") \
+                    else nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h)
+                for k, bit in names.items():
+                    if r & bit:
+                        self.reasons.add(k)
+            except Exception:
+                pass
+            time.sleep(0.02)
+
+    def __enter__(self):
+        if self.nv:
+            self.t.start()
+        return self
+
+    def __exit__(self, *a):
+        self._stop.set()
+        if self.nv:
+            self.t.join()
+
+    def summary(self):
+        if not self.samples:
+            return {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": ["unavailable"]}
+        return {"sm_mhz": statistics.median(self.samples), "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons)}
+
+
+# ------------------------------------------------------------------------------ CPU oracle
+
+class OracleWorkload:
+    """The same step on the CPU oracle, as it stands (numpy fp64)."""
+
+    def __init__(self, cache_len):
+        from oracle import ouroboros as ob, transformer as tf
+        self.ob, self.tf = ob, tf
+        self.m, _, self.P, _ = synth.config("C2")
+        dev = "cuda:0" if torch.cuda.is_available() else "cpu"       # the generator is device independent
+        w = synth.model_weights(self.m, SEED, device=dev)
+        self.W = tf.Weights(self.m, w)
+        k, v = synth.kv_fill(self.m, SEED + 1, cache_len, device=dev)
+        self.cache = tf.KVCache(self.m, k.double().cpu().numpy(), v.double().cpu().numpy(), cache_len)
+        self.L = cache_len
+        self.draft, self.grams = block_inputs(self.m, self.P)
+        self.pool = ob.PhrasePool(self.P.pool_sets, self.P.pool_ways, self.P.beta)
+        for g in self.grams:
+            self.pool.insert(g)
+        self.bytes = algorithmic_bytes(self.m, self.P.block_max, cache_len)
+
+    def step(self):
+        ob, tf, P = self.ob, self.tf, self.P
+        self.cache.length = self.L
+        d = self.draft.tolist()
+        cands = self.pool.lookup(d[-1], P.K)
+        tokens, pos, group, vis = ob.build_block(self.L, PENDING, d, cands)
+        o = tf.argmax_rows(tf.forward(self.W, self.cache, tokens, pos, vis))
+        A, j, m, acc = ob.accept(tokens, o, P.gamma, P.S, len(cands))
+        ob.compact(self.cache, self.L, P.gamma, P.S, A, j, m)
+        seq = [0] * self.L + [PENDING] + acc
+        self.pool.apply(ob.harvest_ops(tokens, o, P.gamma, P.S, len(cands), A, seq, len(acc), P))
+        return acc
+
+
+def blas_threads():
+    try:
+        from threadpoolctl import threadpool_info
+        n = [i.get("num_threads", 0) for i in threadpool_info() if i.get("user_api") == "blas"]
+        return max(n) if n else os.cpu_count()
+    except Exception:
+        return os.cpu_count()
+
+
+def time_oracle(cache_len, budget_s, max_steps=None):
+    wl = OracleWorkload(cache_len)
+    wl.step()
+    t0 = time.perf_counter()
+    n = 0
+    while True:
+        wl.step()
+        n += 1
+        el = time.perf_counter() - t0
+        if el > budget_s or (max_steps and n >= max_steps):
+            break
+    return wl.bytes["total"] * n / el / 1e9, n, el
+
+
+# ----------------------------------------------------------------------------------- main
+
+def run_reference(args, rank):
+    if rank != 0:
+        return
+    total = args.steps + args.warmup
+    gbs, n, el = time_oracle(args.cache_len, 150.0 * args.steps / max(1, total), max_steps=args.steps)
+    cores = blas_threads()
+    sample = f"{n} of {args.steps} steps of the full workload executed ({el:.1f} s), rate taken over those"
+    line = {"impl": "reference", "metric": METRIC, "value": gbs, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": el / n * 1e3, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": workload_config(args.cache_len),
+            "cpu_baseline": {"value": gbs, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+            "e2e": {"value": gbs, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line))
+
+
+def workload_config(cache_len):
+    return {"workload": "configs[1]: one 7B-shaped decoder layer + LM head, bf16, verify block of 37 rows "
+                        "(1 + 4 draft + 4 phrases x 8)", "cache_len": cache_len, "block_rows": 37, "gamma": 4, "beta": 9,
+            "K": 4, "vocab": 32000, "l2": "inputs (734 MB per step) larger than L2, each byte read once per step",
+            "parallelism": "replicas"}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=2000)
+    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--cache-len", type=int, default=4096)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if args.impl == "reference":
+        return run_reference(args, rank)
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU path); use --impl reference for the oracle")
+    from paper_2402_13720_b200 import binding, dist_util
+    torch.cuda.set_device(local)
+    device = f"cuda:{local}"
+    group = dist_util.init(world, rank, "nccl") if world > 1 else None
+    wl = GpuWorkload(device, args.cache_len)
+    lib = binding.lib()
+    for _ in range(max(3, args.warmup)):
+        wl.check()
+    stream = torch.cuda.current_stream()
+
+    def timed(host_inputs):
+        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        dist_util.barrier(group)
+        torch.cuda.synchronize()
+        launches0 = lib.ouro_kernel_launches()
+        with ClockSampler(local) as cs:
+            ev0.record(stream)
+            for _ in range(args.steps):
+                wl.step(host_inputs)
+            ev1.record(stream)
+            torch.cuda.synchronize()
+        dist_util.barrier(group)
+        ms = dist_util.max_over_ranks(ev0.elapsed_time(ev1), group)
+        return ms, lib.ouro_kernel_launches() - launches0, cs.summary()
+
+    ms, launches, clocks = timed(False)
+    ms_e2e, _, _ = timed(True)
+    total_bytes = dist_util.sum_over_ranks(wl.bytes["total"] * args.steps, group)   # every replica's units
+    value = total_bytes / (ms * 1e-3) / 1e9
+    e2e = total_bytes / (ms_e2e * 1e-3) / 1e9
+
+    # per-kernel-class device time of the forward, events on the library's own stream
+    prof = {}
+    psteps = min(args.steps, 200)
+    for cls in PROF_CLASSES + ("forward",):
+        wl.eng.profile_enable(cls)
+        for _ in range(psteps):
+            wl.step()
+        t, n = wl.eng.profile_read()
+        prof[cls] = (t / max(1, n), n // psteps)
+    wl.eng.profile_enable("off")
+    peaks = {}
+    try:
+        peaks = json.load(open(os.path.join(ROOT, "MEASURED_PEAKS.json")))
+    except Exception:
+        pass
+    peak, peak_kind = (peaks["hbm_gbs"], "measured") if "hbm_gbs" in peaks else (6650.0, "fallback")
+    dom = max(PROF_CLASSES, key=lambda c: prof[c][0] * prof[c][1])
+    dom_ms = prof[dom][0]
+    achieved = wl.bytes["per_class"][dom] / (dom_ms * 1e-3) / 1e9 if dom_ms > 0 else 0.0
+    fwd_ms = prof["forward"][0]
+    roofline = {"bound": "hbm", "kernel": dom, "achieved": achieved, "peak": peak, "peak_kind": peak_kind, "unit": "GB/s",
+                "frac": achieved / peak, "traffic": None,
+                "kernel_us": {c: round(prof[c][0] * 1e3, 2) for c in PROF_CLASSES},
+                "forward_us": round(fwd_ms * 1e3, 2),
+                "forward_gbs": wl.bytes["total"] / (fwd_ms * 1e-3) / 1e9 if fwd_ms > 0 else 0.0,
+                "forward_frac": wl.bytes["total"] / (fwd_ms * 1e-3) / 1e9 / peak if fwd_ms > 0 else 0.0}
+    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(3, args.warmup),
+            "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
+            "data": "synthetic", "config": workload_config(args.cache_len), "clocks": clocks,
+            "e2e": {"value": e2e, "unit": UNIT, "h2d_bytes_per_step": int(wl.draft.nbytes),
+                    "d2h_bytes_per_step": 216},   # acceptance record (212 B) + block row count (4 B)
+            "gpu_launches": int(launches), "roofline": roofline, "bytes_per_step": wl.bytes["total"]}
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        gbs, n, el = time_oracle(args.cache_len, 10.0)
+        line["cpu_baseline"] = {"value": gbs, "unit": UNIT, "cores": blas_threads(), "kind": "oracle",
+                                "sample": f"{n} full steps of the same workload in {el:.1f} s"}
+    if rank == 0:
+        print(json.dumps(line))
+    dist_util.finish(group)
+
+
+if __name__ == "__main__":
+    main()

@@ -190,6 +190,21 @@ int ouro_generate(ouro_ctx *ctx, const int32_t *prompt_host, int32_t n_prompt, i
 int ouro_generate_vanilla(ouro_ctx *ctx, const int32_t *prompt_host, int32_t n_prompt, int32_t max_new,
                           int32_t *out_host, int32_t *n_out, ouro_stats *stats_or_null);
 
+/* Measurement aid (no counterpart in the paper, which reports end-to-end speed only): while enabled,
+ * every launch of the kernel class `kernel_class` inside ouro_verify_forward is bracketed by CUDA events
+ * on the context's stream.  ouro_profile_read synchronises, adds up the event times and returns the total
+ * milliseconds and the number of launches since the last ouro_profile_enable.  Other kernels are not
+ * touched; the extra event records cost about a microsecond per launch, so enable it outside timed runs. */
+enum {
+  OURO_PROF_OFF = -1, OURO_PROF_EMBED = 0, OURO_PROF_NORM = 1, OURO_PROF_QKV = 2, OURO_PROF_ROPE = 3,
+  OURO_PROF_ATTENTION = 4, OURO_PROF_WO = 5, OURO_PROF_GATEUP = 6, OURO_PROF_DOWN = 7, OURO_PROF_HEAD = 8,
+  OURO_PROF_ARGMAX = 9, OURO_PROF_FORWARD = 10 /* the whole forward */
+};
+/* Number of kernels this library has launched in this process (all contexts), for launch accounting. */
+uint64_t ouro_kernel_launches(void);
+int ouro_profile_enable(ouro_ctx *ctx, int kernel_class);
+int ouro_profile_read(ouro_ctx *ctx, float *ms_total, int32_t *launches);
+
 #ifdef __cplusplus
 }
 #endif

@@ -76,6 +76,9 @@ _SIGNATURES = {
     "ouro_accept_and_compact": (C.c_int, [C.c_void_p, C.c_void_p, _I32P, _I32P, _I32P, _I32P]),
     "ouro_advance": (C.c_int, [C.c_void_p, C.c_int, C.c_int32]),
     "ouro_draft": (C.c_int, [C.c_void_p, C.c_void_p]),
+    "ouro_kernel_launches": (C.c_uint64, []),
+    "ouro_profile_enable": (C.c_int, [C.c_void_p, C.c_int]),
+    "ouro_profile_read": (C.c_int, [C.c_void_p, _F32P, _I32P]),
     "ouro_generate": (C.c_int, [C.c_void_p, _I32P, C.c_int32, C.c_int32, C.c_int32, _I32P, _I32P, C.POINTER(StatsC)]),
     "ouro_generate_vanilla": (C.c_int, [C.c_void_p, _I32P, C.c_int32, C.c_int32, _I32P, _I32P, C.POINTER(StatsC)]),
 }
@@ -296,6 +299,17 @@ class Engine:
 
     def advance(self, which, n):
         self._ck(self.L.ouro_advance(self.ctx, which, n))
+
+    # ---- measurement -------------------------------------------------------------------------
+    PROF = dict(off=-1, embed=0, norm=1, qkv=2, rope=3, attention=4, wo=5, gateup=6, down=7, head=8, argmax=9, forward=10)
+
+    def profile_enable(self, kernel_class):
+        self._ck(self.L.ouro_profile_enable(self.ctx, self.PROF[kernel_class] if isinstance(kernel_class, str) else kernel_class))
+
+    def profile_read(self):
+        ms, n = C.c_float(), C.c_int32()
+        self._ck(self.L.ouro_profile_read(self.ctx, C.byref(ms), C.byref(n)))
+        return ms.value, n.value
 
     # ---- loops -------------------------------------------------------------------------------
     def generate(self, prompt, max_new, keep_pool=False):

@@ -8,6 +8,8 @@
 #include "ouro_internal.h"
 
 static thread_local std::string g_create_err;
+unsigned long long g_ouro_launches = 0;
+extern "C" uint64_t ouro_kernel_launches(void) { return g_ouro_launches; }
 
 static int fail(ouro_ctx *c, int code, const std::string &msg) {
   if (c) c->err = msg; else g_create_err = msg;
@@ -221,6 +223,7 @@ extern "C" int ouro_destroy(ouro_ctx *c) {
   cudaStreamSynchronize(c->stream);
   if (c->pin) cudaFreeHost(c->pin);
   for (auto &e : c->ev) if (e) cudaEventDestroy(e);
+  for (auto &e : c->prof_ev) cudaEventDestroy(e);
   delete c;
   return OURO_OK;
 }
@@ -325,6 +328,45 @@ extern "C" int ouro_block_get(ouro_ctx *c, int which, int32_t *tok, int32_t *pos
   return OURO_OK;
 }
 
+// --------------------------------------------------------------------------------- profiling
+static void prof_flush(ouro_ctx *c) {
+  if (c->prof_used == 0) return;
+  cudaEventSynchronize(c->prof_ev[c->prof_used - 1]);
+  for (size_t i = 0; i + 1 < c->prof_used; i += 2) {
+    float ms = 0.f;
+    if (cudaEventElapsedTime(&ms, c->prof_ev[i], c->prof_ev[i + 1]) == cudaSuccess) c->prof_ms += ms;
+    c->prof_launches += 1;
+  }
+  c->prof_used = 0;
+}
+void prof_mark(ouro_ctx *c, int) {
+  if (c->prof_used == c->prof_ev.size()) {
+    if (c->prof_ev.size() >= 512) {
+      prof_flush(c);
+    } else {
+      cudaEvent_t e;
+      if (cudaEventCreate(&e) != cudaSuccess) return;
+      c->prof_ev.push_back(e);
+    }
+  }
+  cudaEventRecord(c->prof_ev[c->prof_used++], c->stream);
+}
+extern "C" int ouro_profile_enable(ouro_ctx *c, int kernel_class) {
+  if (!c || kernel_class < OURO_PROF_OFF || kernel_class > OURO_PROF_FORWARD) return OURO_EINVAL;
+  prof_flush(c);
+  c->prof_class = kernel_class;
+  c->prof_ms = 0.0;
+  c->prof_launches = 0;
+  return OURO_OK;
+}
+extern "C" int ouro_profile_read(ouro_ctx *c, float *ms_total, int32_t *launches) {
+  if (!c) return OURO_EINVAL;
+  prof_flush(c);
+  if (ms_total) *ms_total = (float)c->prof_ms;
+  if (launches) *launches = (int32_t)c->prof_launches;
+  return OURO_OK;
+}
+
 // ----------------------------------------------------------------------------------- forward
 int ouro_fast_layer(ouro_ctx *c, int which, int layer, int rows);          // tensor-core layer; OURO_ESTATE = not available
 int ouro_fast_head(ouro_ctx *c, int which, int rows, float *logits);      // tensor-core LM head
@@ -338,32 +380,44 @@ static int forward(ouro_ctx *c, int which, int32_t *argmax_dev, float *logits_de
   const int dt = d.dtype, dq = d.n_heads * d.head_dim, dkv = d.n_kv_heads * d.head_dim;
   cudaStream_t s = c->stream;
   Activations &a = c->a;
-  launch_embed(dt, M.embed, M.blk.tok, rows, d.d_model, a.x, s);
+  ProfScope whole(c, OURO_PROF_FORWARD);
+  { ProfScope ps(c, OURO_PROF_EMBED); launch_embed(dt, M.embed, M.blk.tok, rows, d.d_model, a.x, s); }
   for (int l = 0; l < d.n_layers; ++l) {
     int rc = ouro_fast_layer(c, which, l, rows);
     if (rc == OURO_OK) continue;
     if (rc != OURO_ESTATE) return rc;
-    launch_rmsnorm(dt, a.x, M.attn_norm[l], rows, d.d_model, d.rms_eps, a.xn, s);
-    GemmSegs qkv{{M.wq[l], M.wk[l], M.wv[l]}, {dq, dkv, dkv}, 3};
-    launch_gemm_simple(dt, a.xn, qkv, rows, d.d_model, a.qkv, dq + 2 * dkv, EPI_STORE, s);
-    launch_rope_append(d, a.qkv, M.blk.pos, M.rope_cos, M.rope_sin, rows, L, l, a.q, M.k_cache, M.v_cache, s);
-    launch_attention_simple(d, a.q, M.k_cache, M.v_cache, M.blk, rows, l, a.att, s);
-    GemmSegs wo{{M.wo[l], nullptr, nullptr}, {d.d_model, 0, 0}, 1};
-    launch_gemm_simple(dt, a.att, wo, rows, dq, a.x, d.d_model, EPI_RESIDUAL, s);
-    launch_rmsnorm(dt, a.x, M.ffn_norm[l], rows, d.d_model, d.rms_eps, a.xn, s);
-    launch_gemm_swiglu_simple(dt, a.xn, M.w_gate[l], M.w_up[l], rows, d.d_model, d.d_ffn, a.act, s);
-    GemmSegs wd{{M.w_down[l], nullptr, nullptr}, {d.d_model, 0, 0}, 1};
-    launch_gemm_simple(dt, a.act, wd, rows, d.d_ffn, a.x, d.d_model, EPI_RESIDUAL, s);
+    { ProfScope ps(c, OURO_PROF_NORM); launch_rmsnorm(dt, a.x, M.attn_norm[l], rows, d.d_model, d.rms_eps, a.xn, s); }
+    {
+      ProfScope ps(c, OURO_PROF_QKV);
+      GemmSegs qkv{{M.wq[l], M.wk[l], M.wv[l]}, {dq, dkv, dkv}, 3};
+      launch_gemm_simple(dt, a.xn, qkv, rows, d.d_model, a.qkv, dq + 2 * dkv, EPI_STORE, s);
+    }
+    { ProfScope ps(c, OURO_PROF_ROPE); launch_rope_append(d, a.qkv, M.blk.pos, M.rope_cos, M.rope_sin, rows, L, l, a.q, M.k_cache, M.v_cache, s); }
+    { ProfScope ps(c, OURO_PROF_ATTENTION); launch_attention_simple(d, a.q, M.k_cache, M.v_cache, M.blk, rows, l, a.att, s); }
+    {
+      ProfScope ps(c, OURO_PROF_WO);
+      GemmSegs wo{{M.wo[l], nullptr, nullptr}, {d.d_model, 0, 0}, 1};
+      launch_gemm_simple(dt, a.att, wo, rows, dq, a.x, d.d_model, EPI_RESIDUAL, s);
+    }
+    { ProfScope ps(c, OURO_PROF_NORM); launch_rmsnorm(dt, a.x, M.ffn_norm[l], rows, d.d_model, d.rms_eps, a.xn, s); }
+    { ProfScope ps(c, OURO_PROF_GATEUP); launch_gemm_swiglu_simple(dt, a.xn, M.w_gate[l], M.w_up[l], rows, d.d_model, d.d_ffn, a.act, s); }
+    {
+      ProfScope ps(c, OURO_PROF_DOWN);
+      GemmSegs wd{{M.w_down[l], nullptr, nullptr}, {d.d_model, 0, 0}, 1};
+      launch_gemm_simple(dt, a.act, wd, rows, d.d_ffn, a.x, d.d_model, EPI_RESIDUAL, s);
+    }
   }
   float *logits = logits_dev ? logits_dev : a.logits;
   int rc = ouro_fast_head(c, which, rows, logits);
   if (rc == OURO_ESTATE) {
-    launch_rmsnorm(dt, a.x, M.final_norm, rows, d.d_model, d.rms_eps, a.xn, s);
+    { ProfScope ps(c, OURO_PROF_NORM); launch_rmsnorm(dt, a.x, M.final_norm, rows, d.d_model, d.rms_eps, a.xn, s); }
+    ProfScope ps(c, OURO_PROF_HEAD);
     GemmSegs head{{M.lm_head, nullptr, nullptr}, {d.vocab, 0, 0}, 1};
     launch_gemm_simple(dt, a.xn, head, rows, d.d_model, logits, d.vocab, EPI_STORE, s);
   } else if (rc != OURO_OK) {
     return rc;
   }
+  ProfScope pa(c, OURO_PROF_ARGMAX);
   launch_argmax(logits, rows, d.vocab, argmax_dev, s);
   CKL();
   return OURO_OK;

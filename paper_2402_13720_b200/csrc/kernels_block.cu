@@ -135,16 +135,20 @@ __global__ void pool_update_kernel(PoolDev P, DevState *st, const int32_t *ngram
 }
 
 void launch_pool_clear(const PoolDev &P, DevState *st, cudaStream_t s) {
+  OURO_COUNT_LAUNCH();
   int n = P.sets * P.ways;
   pool_clear_kernel<<<(n + 255) / 256, 256, 0, s>>>(P, st);
 }
 void launch_pool_lookup(const PoolDev &P, const int32_t *key_dev, int key_index, int32_t key_value, int K,
                         int32_t *suffix, int32_t *count, cudaStream_t s) {
+  OURO_COUNT_LAUNCH();
   pool_lookup_kernel<<<1, 32, 0, s>>>(P, key_dev, key_index, key_value, K, suffix, count);
 }
 void launch_pool_update(const PoolDev &P, DevState *st, const int32_t *ngrams, int n, int beta, int stride,
                         cudaStream_t s) {
-  if (n > 0) pool_update_kernel<<<1, 32, 0, s>>>(P, st, ngrams, n, beta, stride);
+  if (n <= 0) return;
+  OURO_COUNT_LAUNCH();
+  pool_update_kernel<<<1, 32, 0, s>>>(P, st, ngrams, n, beta, stride);
 }
 
 // --------------------------------------------------------------------------- candidate packing
@@ -202,9 +206,11 @@ __global__ void assemble_causal_kernel(BlockDev b, const int32_t *tokens, int n,
 
 void launch_assemble_candidates(const BlockDev &b, DevState *st, const int32_t *draft, const int32_t *suffix,
                                 const int32_t *count, int L, int gamma, int S, int K, cudaStream_t s) {
+  OURO_COUNT_LAUNCH();
   assemble_candidates_kernel<<<1, OURO_MAX_ROWS, 0, s>>>(b, st, draft, suffix, count, L, gamma, S, K);
 }
 void launch_assemble_causal(const BlockDev &b, const int32_t *tokens, int n, int L, cudaStream_t s) {
+  OURO_COUNT_LAUNCH();
   assemble_causal_kernel<<<1, OURO_MAX_ROWS, 0, s>>>(b, tokens, n, L);
 }
 
@@ -251,6 +257,7 @@ __global__ void accept_kernel(BlockDev b, DevState *st, const int32_t *o, int32_
 
 void launch_accept(const BlockDev &b, DevState *st, const int32_t *o, int32_t *seq_dev, int gamma, int S,
                    cudaStream_t s) {
+  OURO_COUNT_LAUNCH();
   accept_kernel<<<1, 32, 0, s>>>(b, st, o, seq_dev, gamma, S);
 }
 
@@ -273,6 +280,7 @@ __global__ void compact_kernel(T *k_cache, T *v_cache, const DevState *st, int L
 void launch_compact(const ouro_model_desc &d, void *k_cache, void *v_cache, const DevState *st, int L, int gamma,
                     int S, cudaStream_t s) {
   if (S <= 0) return;
+  OURO_COUNT_LAUNCH();
   dim3 grid(S, d.n_layers * 2);
   int d_kv = d.n_kv_heads * d.head_dim;
   if (d.dtype == OURO_BF16)
@@ -334,6 +342,7 @@ __global__ void harvest_kernel(BlockDev b, DevState *st, PoolDev P, const int32_
 
 void launch_harvest(const BlockDev &b, DevState *st, const PoolDev &P, const int32_t *o, const int32_t *seq_dev,
                     int gamma, int S, unsigned flags, cudaStream_t s) {
+  OURO_COUNT_LAUNCH();
   harvest_kernel<<<1, 32, 0, s>>>(b, st, P, o, seq_dev, gamma, S, flags);
 }
 
@@ -373,6 +382,7 @@ __global__ void argmax_kernel(const float *logits, int vocab, int32_t *out) {
 }
 
 void launch_argmax(const float *logits, int rows, int vocab, int32_t *out, cudaStream_t s) {
+  OURO_COUNT_LAUNCH();
   argmax_kernel<<<rows, 256, 0, s>>>(logits, vocab, out);
 }
 
@@ -383,11 +393,13 @@ __global__ void vanilla_accept_kernel(DevState *st, const int32_t *o, int32_t *s
   st->n_seq += 1;
 }
 void launch_vanilla_accept(DevState *st, const int32_t *o, int32_t *seq_dev, cudaStream_t s) {
+  OURO_COUNT_LAUNCH();
   vanilla_accept_kernel<<<1, 1, 0, s>>>(st, o, seq_dev);
 }
 
 __global__ void pick_token_kernel(const int32_t *src, int index, int32_t *dst) { *dst = src[index]; }
 void launch_pick_token(const int32_t *src, int index, int32_t *dst, cudaStream_t s) {
+  OURO_COUNT_LAUNCH();
   pick_token_kernel<<<1, 1, 0, s>>>(src, index, dst);
 }
 
@@ -405,5 +417,6 @@ __global__ void set_state_kernel(DevState *st, int32_t *seq_dev, int n_seq, int 
   }
 }
 void launch_set_state(DevState *st, int32_t *seq_dev, int n_seq, int pending, int fill, cudaStream_t s) {
+  OURO_COUNT_LAUNCH();
   set_state_kernel<<<8, 256, 0, s>>>(st, seq_dev, n_seq, pending, fill);
 }

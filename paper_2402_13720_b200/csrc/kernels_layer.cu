@@ -57,6 +57,7 @@ __global__ void rope_table_kernel(float *cos_t, float *sin_t, int max_seq, int h
   sin_t[idx] = (float)sin(ang);
 }
 void launch_rope_table(float *cos_t, float *sin_t, int max_seq, int head_dim, float theta, cudaStream_t s) {
+  OURO_COUNT_LAUNCH();
   int n = max_seq * (head_dim / 2);
   rope_table_kernel<<<(n + 255) / 256, 256, 0, s>>>(cos_t, sin_t, max_seq, head_dim / 2, (double)theta);
 }
@@ -69,6 +70,7 @@ __global__ void embed_kernel(const T *E, const int32_t *tok, int d, float *x) {
   for (int i = threadIdx.x; i < d; i += blockDim.x) dst[i] = to_f<T>(src[i]);
 }
 void launch_embed(int dtype, const void *E, const int32_t *tok, int rows, int d, float *x, cudaStream_t s) {
+  OURO_COUNT_LAUNCH();
   if (dtype == OURO_BF16) embed_kernel<__nv_bfloat16><<<rows, 256, 0, s>>>((const __nv_bfloat16 *)E, tok, d, x);
   else embed_kernel<float><<<rows, 256, 0, s>>>((const float *)E, tok, d, x);
 }
@@ -91,6 +93,7 @@ __global__ void rmsnorm_kernel(const float *x, const T *g, int d, float eps, T *
   for (int i = threadIdx.x; i < d; i += blockDim.x) o[i] = from_f<T>(to_f<T>(g[i]) * (row[i] * inv));
 }
 void launch_rmsnorm(int dtype, const float *x, const void *g, int rows, int d, float eps, void *out, cudaStream_t s) {
+  OURO_COUNT_LAUNCH();
   if (dtype == OURO_BF16)
     rmsnorm_kernel<__nv_bfloat16><<<rows, 256, 0, s>>>(x, (const __nv_bfloat16 *)g, d, eps, (__nv_bfloat16 *)out);
   else rmsnorm_kernel<float><<<rows, 256, 0, s>>>(x, (const float *)g, d, eps, (float *)out);
@@ -146,6 +149,7 @@ __global__ void gemm_simple_kernel(const T *X, GemmSegs W, int rows, int K, floa
 }
 void launch_gemm_simple(int dtype, const void *X, const GemmSegs &W, int rows, int K, float *Y, int ldy, int epi,
                         cudaStream_t s) {
+  OURO_COUNT_LAUNCH();
   int ntot = 0;
   for (int i = 0; i < W.count; ++i) ntot += W.n[i];
   int grid = (ntot + 3) / 4;
@@ -172,6 +176,7 @@ __global__ void gemm_swiglu_simple_kernel(const T *X, const T *Wg, const T *Wu, 
 }
 void launch_gemm_swiglu_simple(int dtype, const void *X, const void *Wg, const void *Wu, int rows, int K, int F,
                                void *act, cudaStream_t s) {
+  OURO_COUNT_LAUNCH();
   int grid = (F + 3) / 4;
   if (dtype == OURO_BF16)
     gemm_swiglu_simple_kernel<__nv_bfloat16><<<grid, 128, 0, s>>>((const __nv_bfloat16 *)X, (const __nv_bfloat16 *)Wg,
@@ -205,6 +210,7 @@ __global__ void rope_append_kernel(const float *qkv, const int32_t *pos, const f
 void launch_rope_append(const ouro_model_desc &d, const float *qkv, const int32_t *pos, const float *cos_t,
                         const float *sin_t, int rows, int L, int layer, void *q, void *k_cache, void *v_cache,
                         cudaStream_t s) {
+  OURO_COUNT_LAUNCH();
   size_t off = (size_t)layer * d.max_seq * d.n_kv_heads * d.head_dim;
   if (d.dtype == OURO_BF16)
     rope_append_kernel<__nv_bfloat16><<<rows, 256, 0, s>>>(qkv, pos, cos_t, sin_t, d.n_heads, d.n_kv_heads, d.head_dim, L,
@@ -275,6 +281,7 @@ __global__ void attention_simple_kernel(const T *q, const T *k_cache, const T *v
 }
 void launch_attention_simple(const ouro_model_desc &d, const void *q, const void *k_cache, const void *v_cache,
                              const BlockDev &b, int rows, int layer, void *out, cudaStream_t s) {
+  OURO_COUNT_LAUNCH();
   size_t off = (size_t)layer * d.max_seq * d.n_kv_heads * d.head_dim;
   int warps = 4;
   dim3 grid(rows, (d.n_heads + warps - 1) / warps);

@@ -12,6 +12,9 @@
 
 typedef unsigned long long u64;
 
+extern unsigned long long g_ouro_launches;   // kernels launched by this library since it was loaded
+#define OURO_COUNT_LAUNCH() (++g_ouro_launches)
+
 // Device-resident scalars of one decoding stream.
 struct DevState {
   int32_t pending;   // last accepted token; its K/V is not cached yet (block row 0 of the next step)
@@ -91,6 +94,18 @@ struct ouro_ctx {
   int32_t step = 0;
   std::string err;
   cudaEvent_t ev[6] = {nullptr, nullptr, nullptr, nullptr, nullptr, nullptr};
+  // per-kernel-class timing (ouro_profile_*)
+  int prof_class = -1;
+  std::vector<cudaEvent_t> prof_ev;
+  size_t prof_used = 0;
+  double prof_ms = 0.0;
+  long prof_launches = 0;
+};
+void prof_mark(ouro_ctx *c, int kernel_class);   // call before and after the launches of a class
+struct ProfScope {
+  ouro_ctx *c; int k;
+  ProfScope(ouro_ctx *c_, int k_) : c(c_), k(k_) { if (c->prof_class == k) prof_mark(c, k); }
+  ~ProfScope() { if (c->prof_class == k) prof_mark(c, k); }
 };
 enum { PIN_INTS = 1024 };
 
