@@ -95,8 +95,12 @@ class GpuWorkload:
         return e.accept_and_compact()                 # returns host values: a device->host read per step
 
     def check(self):
-        n, chosen, A, acc = self.step()
-        assert self.eng.block_get()[0].shape[0] == self.B, "the pool no longer yields K candidates"
+        e = self.eng
+        e.set_state(self.L, PENDING)
+        e.assemble_candidates()
+        assert e.block_get()[0].shape[0] == self.B, "the pool no longer yields K candidates"
+        e.verify_forward()
+        n, chosen, A, acc = e.accept_and_compact()
         assert 1 <= n <= self.P.gamma + self.P.beta
         return n
 
