@@ -196,6 +196,7 @@ extern "C" int ouro_create(const ouro_model_desc *t, const ouro_model_mem *tm, c
     g_create_err = msg;
     if (n->pin) cudaFreeHost(n->pin);
     for (auto &e : n->ev) if (e) cudaEventDestroy(e);
+    ouro_fast_teardown(n);
     delete n;
     return code;
   };
@@ -224,6 +225,7 @@ extern "C" int ouro_destroy(ouro_ctx *c) {
   if (c->pin) cudaFreeHost(c->pin);
   for (auto &e : c->ev) if (e) cudaEventDestroy(e);
   for (auto &e : c->prof_ev) cudaEventDestroy(e);
+  ouro_fast_teardown(c);
   delete c;
   return OURO_OK;
 }

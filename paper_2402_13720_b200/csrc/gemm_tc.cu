@@ -1,0 +1,627 @@
+// Weight-streaming GEMM for a few dozen tokens on sm_100a tensor cores (tcgen05 + TMEM), fed by TMA.
+//
+//   Y[t, n] = sum_k X[t, k] * W[n, k]      X: [rows <= 128, K] bf16 activations, W: [N, K] bf16 weights
+//
+// The verification forward is bound by the one pass over the weights (the paper's premise: checking dozens
+// of tokens costs about as much as one, Section 3.2), so the kernel is organised around the weight stream:
+//   * operands are swapped: a 128-row slab of W is the MMA's M side, the tokens (padded to a multiple of 16)
+//     are its N side; the fp32 accumulator [128 x T] lives in TMEM;
+//   * one persistent CTA per SM; the (tile, k-block) iteration space is cut into equal contiguous spans
+//     (stream-K), so every SM streams the same number of bytes whatever N and K are;
+//   * a span that covers only part of a tile's K range leaves a partial tile in scratch memory; the CTA that
+//     arrives last at the tile's counter adds the partials in ascending K order and runs the epilogue.
+//     Nobody waits for anybody, and the result does not depend on arrival order;
+//   * warp 0 issues TMA loads into a ring of shared-memory stages (128-byte swizzle), warp 1 issues
+//     tcgen05.mma and releases stages with tcgen05.commit, warps 2-5 drain TMEM (double buffered) and run the
+//     epilogue: plain store, residual add, or SiLU(gate)*up for the stacked gate/up matrices.
+// The span boundaries depend on N, K and the grid only, never on the number of rows, and an output element
+// is a function of its own row of X: a token's result is bitwise the same in a 1-row and in a 128-row call.
+// Every mbarrier wait is bounded; on expiry the CTA raises the context's status word and drains.
+#include <cuda.h>
+
+#include "ouro_internal.h"
+
+namespace {
+
+constexpr int TILE_N = 128;       // weight rows per tile (MMA M)
+constexpr int BLOCK_K = 64;       // bf16 elements per k-block: one 128-byte swizzle row
+constexpr int A_BYTES = TILE_N * BLOCK_K * 2;
+constexpr int THREADS = 192;      // warp 0 TMA, warp 1 MMA, warps 2..5 epilogue
+constexpr int MAX_GRID = 160;
+constexpr int SLOT_FLOATS = TILE_N * OURO_MAX_ROWS;
+constexpr uint32_t SPIN_LIMIT = 1u << 24;
+constexpr unsigned long long HINT_EVICT_FIRST = 0x12F0000000000000ull;
+constexpr unsigned long long HINT_EVICT_LAST = 0x14F0000000000000ull;
+
+enum { MODE_STORE = 0, MODE_RESIDUAL = 1, MODE_SWIGLU = 2 };
+
+struct GemmParams {
+  CUtensorMap a[3];   // weight matrices stacked along the output dimension (q|k|v), or gate and up
+  CUtensorMap b;      // activations, box = 64 x 16
+  int a_tiles[3];     // tiles of each stacked matrix (MODE_STORE / MODE_RESIDUAL)
+  int a_rows[3];      // output features of each stacked matrix
+  int a_count;
+  int mode;
+  int tiles;          // total tiles
+  int kb;             // k-blocks per tile (K / 64)
+  int t_pad;          // tokens padded to a multiple of 16 (MMA N)
+  int rows;           // valid tokens
+  int stages;
+  float *out_f32;     // MODE_STORE / MODE_RESIDUAL: [rows, ldo]
+  int ldo;
+  __nv_bfloat16 *out_bf16;  // MODE_SWIGLU: [rows, F]
+  float *scratch;     // [grid][2][t][128] partial tiles
+  int *counters;      // [tiles], zero between launches
+  int *status;        // context status word
+};
+
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint64_t *bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint64_t *bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t *bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+// Bounded wait: false when the limit ran out (the caller raises the status word and drains).
+__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity) {
+  uint32_t addr = smem_u32(bar);
+  for (uint32_t i = 0; i < SPIN_LIMIT; ++i) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(addr), "r"(parity)
+        : "memory");
+    if (ok) return true;
+  }
+  return false;
+}
+__device__ __forceinline__ void tma_load_2d(void *dst, const CUtensorMap *map, uint64_t *bar, int x, int y,
+                                            unsigned long long hint) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint"
+      " [%0], [%1, {%3, %4}], [%2], %5;" ::"r"(smem_u32(dst)),
+      "l"(map), "r"(smem_u32(bar)), "r"(x), "r"(y), "l"(hint)
+      : "memory");
+}
+__device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t addr) {
+  // K-major operand in 128-byte swizzle: rows of 128 bytes, 8-row groups 1024 bytes apart.
+  return (uint64_t)((addr & 0x3FFFF) >> 4) | ((uint64_t)1 << 16) | ((uint64_t)(1024 >> 4) << 32) | ((uint64_t)1 << 46) |
+         ((uint64_t)2 << 61);
+}
+__device__ __forceinline__ void mma_bf16(uint32_t tmem_d, uint64_t da, uint64_t db, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}" ::"r"(tmem_d),
+      "l"(da), "l"(db), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+__device__ __forceinline__ void mma_commit(uint64_t *bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void tmem_ld16(uint32_t addr, float *v) {
+  uint32_t r[16];
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+      : "r"(addr));
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+  for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
+}
+__device__ __forceinline__ void fence_before_sync() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void fence_after_sync() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void epi_barrier() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
+
+struct Span {  // one piece of this CTA's iteration range: k-blocks [kb0, kb1) of `tile`
+  int tile, kb0, kb1, n_contrib, slot;
+};
+
+// Walks the CTA's contiguous share of the (tile, k-block) space; identical in every warp role.
+struct SpanWalker {
+  int it, end, kb, per;
+  __device__ SpanWalker(const GemmParams &p) {
+    int total = p.tiles * p.kb;
+    per = (total + gridDim.x - 1) / gridDim.x;
+    it = min(total, (int)blockIdx.x * per);
+    end = min(total, it + per);
+    kb = p.kb;
+  }
+  __device__ bool next(Span &s) {
+    if (it >= end) return false;
+    s.tile = it / kb;
+    s.kb0 = it - s.tile * kb;
+    s.kb1 = min(kb, s.kb0 + (end - it));
+    int first_owner = (s.tile * kb) / per, last_owner = (s.tile * kb + kb - 1) / per;
+    s.n_contrib = last_owner - first_owner + 1;
+    s.slot = (s.tile * kb <= (int)blockIdx.x * per) ? 0 : 1;   // first or last piece of this CTA
+    it += s.kb1 - s.kb0;
+    return true;
+  }
+};
+
+// Locates a tile: which stacked matrix, its first row there, and the first output column.
+__device__ __forceinline__ void locate(const GemmParams &p, int tile, int &seg, int &row0, int &col0, int &valid) {
+  seg = 0;
+  col0 = 0;
+  int t = tile;
+  while (seg + 1 < p.a_count && t >= p.a_tiles[seg]) {
+    t -= p.a_tiles[seg];
+    col0 += p.a_rows[seg];
+    ++seg;
+  }
+  row0 = t * TILE_N;
+  col0 += row0;
+  valid = min(TILE_N, p.a_rows[seg] - row0);
+}
+
+// Final values of one output row n (this thread) for tokens t0..t0+15.
+__device__ __forceinline__ void store_chunk(const GemmParams &p, int col, bool n_ok, int t0, const float *v) {
+  if (!n_ok) return;
+#pragma unroll
+  for (int i = 0; i < 16; ++i) {
+    int t = t0 + i;
+    if (t < p.rows) {
+      float *y = p.out_f32 + (size_t)t * p.ldo + col;
+      *y = p.mode == MODE_RESIDUAL ? *y + v[i] : v[i];
+    }
+  }
+}
+
+__global__ void __launch_bounds__(THREADS, 1) gemm_tc_kernel(const __grid_constant__ GemmParams p) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t *smem = (uint8_t *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+  const int b_bytes = p.t_pad * BLOCK_K * 2;
+  const int stage_bytes = A_BYTES + b_bytes;
+  uint8_t *ring = smem;
+  float *xchg = (float *)(ring + (size_t)p.stages * stage_bytes);          // [64][t_pad] up values (SwiGLU)
+  uint64_t *bars = (uint64_t *)((uint8_t *)xchg + 64 * OURO_MAX_ROWS * 4);
+  uint64_t *full = bars, *empty = bars + 16, *acc_full = bars + 32, *acc_empty = bars + 34;
+  uint32_t *tmem_base_p = (uint32_t *)(bars + 36);
+  volatile int *abort_flag = (volatile int *)(bars + 37);
+  int *last_flag = (int *)(bars + 38);
+  volatile int *wait_flag = (volatile int *)(bars + 39);   // [2]: outcome of the epilogue's accumulator wait
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int acc_cols = p.t_pad <= 32 ? 32 : p.t_pad <= 64 ? 64 : 128;   // columns per accumulator buffer
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < p.stages; ++s) {
+      mbar_init(&full[s], 1);
+      mbar_init(&empty[s], 1);
+    }
+    for (int a = 0; a < 2; ++a) {
+      mbar_init(&acc_full[a], 1);
+      mbar_init(&acc_empty[a], 4);
+    }
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_base_p)),
+                 "r"((uint32_t)(2 * acc_cols)));
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::);
+  }
+  fence_before_sync();
+  __syncthreads();
+  fence_after_sync();
+  const uint32_t tmem_base = *tmem_base_p;
+
+  if (warp == 0) {
+    // ---------------------------------------------------------------- TMA producer
+    if (lane == 0) {
+      SpanWalker w(p);
+      Span s;
+      uint32_t n = 0;
+      bool ok = true;
+      while (ok && w.next(s)) {
+        int seg, row0, col0, valid;
+        if (p.mode == MODE_SWIGLU) { seg = 0; row0 = s.tile * 64; } else locate(p, s.tile, seg, row0, col0, valid);
+        for (int kb = s.kb0; kb < s.kb1 && ok; ++kb, ++n) {
+          int st = n % p.stages;
+          if (n >= (uint32_t)p.stages) ok = mbar_wait(&empty[st], ((n / p.stages) - 1) & 1) && !*abort_flag;
+          if (!ok) break;
+          uint8_t *sa = ring + (size_t)st * stage_bytes, *sb = sa + A_BYTES;
+          mbar_expect_tx(&full[st], stage_bytes);
+          if (p.mode == MODE_SWIGLU) {
+            tma_load_2d(sa, &p.a[0], &full[st], kb * BLOCK_K, row0, HINT_EVICT_FIRST);
+            tma_load_2d(sa + A_BYTES / 2, &p.a[1], &full[st], kb * BLOCK_K, row0, HINT_EVICT_FIRST);
+          } else {
+            tma_load_2d(sa, &p.a[seg], &full[st], kb * BLOCK_K, row0, HINT_EVICT_FIRST);
+          }
+          for (int r = 0; r < p.t_pad; r += 16)
+            tma_load_2d(sb + r * BLOCK_K * 2, &p.b, &full[st], kb * BLOCK_K, r, HINT_EVICT_LAST);
+        }
+      }
+      if (!ok) { *abort_flag = 1; atomicExch(p.status, 1); }
+    }
+  } else if (warp == 1) {
+    // ---------------------------------------------------------------- MMA issuer
+    if (lane == 0) {
+      const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(p.t_pad >> 3) << 17) | ((uint32_t)(TILE_N >> 4) << 24);
+      SpanWalker w(p);
+      Span s;
+      uint32_t n = 0, item = 0;
+      bool ok = true;
+      while (ok && w.next(s)) {
+        int a = item & 1;
+        if (item >= 2) ok = mbar_wait(&acc_empty[a], ((item >> 1) - 1) & 1) && !*abort_flag;
+        if (!ok) break;
+        fence_after_sync();
+        uint32_t tmem_d = tmem_base + a * acc_cols;
+        for (int kb = s.kb0; kb < s.kb1; ++kb, ++n) {
+          int st = n % p.stages;
+          ok = mbar_wait(&full[st], (n / p.stages) & 1) && !*abort_flag;
+          if (!ok) break;
+          fence_after_sync();
+          uint32_t sa = smem_u32(ring + (size_t)st * stage_bytes), sb = sa + A_BYTES;
+          uint64_t da = smem_desc_sw128(sa), db = smem_desc_sw128(sb);
+#pragma unroll
+          for (int k = 0; k < BLOCK_K / 16; ++k) mma_bf16(tmem_d, da + 2 * k, db + 2 * k, idesc, (kb > s.kb0 || k > 0) ? 1u : 0u);
+          mma_commit(&empty[st]);
+        }
+        if (!ok) break;
+        mma_commit(&acc_full[a]);
+        ++item;
+      }
+      if (!ok) { *abort_flag = 1; atomicExch(p.status, 1); }
+    }
+  } else {
+    // ---------------------------------------------------------------- epilogue warps
+    const int q = warp & 3;                      // TMEM lane quarter this warp may read
+    const int nl = q * 32 + lane;                // row of the tile held by this thread
+    const int et = threadIdx.x - 64;             // 0..127 among the epilogue threads
+    SpanWalker w(p);
+    Span s;
+    uint32_t item = 0;
+    bool ok = true;
+    float v[16];
+    while (w.next(s)) {
+      int a = item & 1;
+      // one thread waits (bounded) and tells the others, so that all 128 leave the loop together
+      if (et == 0) wait_flag[a] = mbar_wait(&acc_full[a], (item >> 1) & 1) && !*abort_flag;
+      epi_barrier();
+      ok = wait_flag[a] != 0;
+      if (!ok) break;
+      fence_after_sync();
+      const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + a * acc_cols;
+      int seg = 0, row0 = 0, col0 = 0, valid = TILE_N;
+      if (p.mode != MODE_SWIGLU) locate(p, s.tile, seg, row0, col0, valid);
+      if (s.n_contrib == 1) {
+        if (p.mode == MODE_SWIGLU) {
+          // rows 0..63 hold gate, rows 64..127 hold up, for output features tile*64 + (nl & 63)
+          const int F = p.a_rows[0];
+          const int feat = s.tile * 64 + (nl & 63);
+          for (int t0 = 0; t0 < p.t_pad; t0 += 16) {
+            tmem_ld16(taddr + t0, v);
+            if (nl >= 64) {
+#pragma unroll
+              for (int i = 0; i < 16; ++i) xchg[(nl - 64) * OURO_MAX_ROWS + t0 + i] = v[i];
+            }
+            epi_barrier();
+            if (nl < 64 && feat < F) {
+#pragma unroll
+              for (int i = 0; i < 16; ++i) {
+                int t = t0 + i;
+                if (t < p.rows) {
+                  float g = v[i], u = xchg[nl * OURO_MAX_ROWS + t];
+                  p.out_bf16[(size_t)t * F + feat] = __float2bfloat16_rn(g / (1.0f + __expf(-g)) * u);
+                }
+              }
+            }
+            epi_barrier();
+          }
+        } else {
+          for (int t0 = 0; t0 < p.t_pad; t0 += 16) {
+            tmem_ld16(taddr + t0, v);
+            store_chunk(p, col0 + nl, nl < valid, t0, v);
+          }
+        }
+        fence_before_sync();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&acc_empty[a]);
+      } else {
+        // partial tile: park it, and let the last arriver of the tile add everything up in K order
+        float *mine = p.scratch + ((size_t)blockIdx.x * 2 + s.slot) * SLOT_FLOATS;
+        for (int t0 = 0; t0 < p.t_pad; t0 += 16) {
+          tmem_ld16(taddr + t0, v);
+#pragma unroll
+          for (int i = 0; i < 16; ++i)
+            if (t0 + i < p.rows) __stcg(mine + (size_t)(t0 + i) * TILE_N + nl, v[i]);
+        }
+        fence_before_sync();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&acc_empty[a]);
+        __threadfence();
+        epi_barrier();
+        if (et == 0) {
+          int old = atomicAdd(p.counters + s.tile, 1);
+          *last_flag = old == s.n_contrib - 1;
+          if (old == s.n_contrib - 1) p.counters[s.tile] = 0;     // ready for the next launch
+        }
+        epi_barrier();
+        const bool last = *last_flag != 0;
+        epi_barrier();
+        if (last) {
+          __threadfence();
+          const int per = w.per;
+          const int first_owner = (s.tile * p.kb) / per;
+          if (p.mode == MODE_SWIGLU) {
+            const int F = p.a_rows[0];
+            // 128 threads: thread -> (feature r = et & 63, token parity et >> 6)
+            const int r = et & 63, feat = s.tile * 64 + r;
+            for (int t = et >> 6; t < p.rows; t += 2) {
+              float g = 0.f, u = 0.f;
+              for (int c = 0; c < s.n_contrib; ++c) {
+                int owner = first_owner + c;
+                int slot = (s.tile * p.kb <= owner * per) ? 0 : 1;
+                const float *src = p.scratch + ((size_t)owner * 2 + slot) * SLOT_FLOATS + (size_t)t * TILE_N;
+                g += __ldcg(src + r);
+                u += __ldcg(src + 64 + r);
+              }
+              if (feat < F) p.out_bf16[(size_t)t * F + feat] = __float2bfloat16_rn(g / (1.0f + __expf(-g)) * u);
+            }
+          } else {
+            for (int t = 0; t < p.rows; ++t) {
+              float acc = 0.f;
+              for (int c = 0; c < s.n_contrib; ++c) {
+                int owner = first_owner + c;
+                int slot = (s.tile * p.kb <= owner * per) ? 0 : 1;
+                acc += __ldcg(p.scratch + ((size_t)owner * 2 + slot) * SLOT_FLOATS + (size_t)t * TILE_N + nl);
+              }
+              if (nl < valid) {
+                float *y = p.out_f32 + (size_t)t * p.ldo + col0 + nl;
+                *y = p.mode == MODE_RESIDUAL ? *y + acc : acc;
+              }
+            }
+          }
+        }
+      }
+      ++item;
+    }
+    if (!ok && et == 0) { *abort_flag = 1; atomicExch(p.status, 1); }
+  }
+  // ------------------------------------------------------------------ teardown
+  fence_before_sync();
+  __syncthreads();
+  if (warp == 1) {
+    fence_after_sync();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)(2 * acc_cols)));
+  }
+}
+
+// ------------------------------------------------------------------------------- host side
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *, const cuuint64_t *,
+                                  const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+EncodeTiledFn g_encode = nullptr;
+
+bool make_map(CUtensorMap *m, const void *base, int rows, int K, int box_rows) {
+  cuuint64_t dims[2] = {(cuuint64_t)K, (cuuint64_t)rows};
+  cuuint64_t strides[1] = {(cuuint64_t)K * 2};
+  cuuint32_t box[2] = {BLOCK_K, (cuuint32_t)box_rows};
+  cuuint32_t es[2] = {1, 1};
+  return g_encode(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(base), dims, strides, box, es,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+struct LayerMaps {
+  CUtensorMap wq, wk, wv, wo, wg, wu, wd;
+};
+struct FastModel {
+  bool ok = false;
+  std::vector<LayerMaps> layers;
+  CUtensorMap head, x_d, x_q, x_f;   // activations: normed [128, d], attention out [128, dq], SwiGLU out [128, F]
+};
+struct FastState {
+  FastModel m[2];
+  int grid = 0;
+  int smem_max = 0;
+  float *slots = nullptr;
+  int *counters = nullptr;
+};
+constexpr int MAX_TILES = 4096;
+
+size_t slots_bytes() { return (size_t)MAX_GRID * 2 * SLOT_FLOATS * sizeof(float); }
+
+int stages_for(int t_pad, int smem_max) {
+  int stage = A_BYTES + t_pad * BLOCK_K * 2;
+  int fixed = 1024 + 64 * OURO_MAX_ROWS * 4 + 512;   // alignment slack, SwiGLU exchange buffer, barriers and flags
+  int s = (smem_max - fixed) / stage;
+  return s > 12 ? 12 : s;
+}
+
+}  // namespace
+
+struct ouro_fast { FastState s; };
+
+size_t ouro_scratch_bytes(const ouro_model_desc *, const ouro_model_desc *) {
+  return slots_bytes() + MAX_TILES * sizeof(int) + 256;
+}
+
+static bool shape_ok(const ouro_model_desc &d) {
+  int dq = d.n_heads * d.head_dim;
+  return d.dtype == OURO_BF16 && d.d_model % 64 == 0 && dq % 64 == 0 && d.d_ffn % 64 == 0 && d.vocab % 8 == 0 &&
+         (d.vocab + TILE_N - 1) / TILE_N <= MAX_TILES && (2 * d.d_ffn + TILE_N - 1) / TILE_N <= MAX_TILES;
+}
+
+int ouro_fast_setup(ouro_ctx *c) {
+  c->fast = nullptr;
+  bool any = false;
+  for (auto &M : c->m) any = any || (M.present && shape_ok(M.d));
+  if (!any) return OURO_OK;
+  int dev = 0, sms = 0, smem = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess ||
+      cudaDeviceGetAttribute(&smem, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev) != cudaSuccess) {
+    c->err = "device attributes unavailable";
+    return OURO_ECUDA;
+  }
+  if (!g_encode) {
+    void *fn = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess || !fn) {
+      c->err = "cuTensorMapEncodeTiled unavailable";
+      return OURO_ECUDA;
+    }
+    g_encode = (EncodeTiledFn)fn;
+  }
+  ouro_fast *f = new ouro_fast();
+  f->s.grid = sms < MAX_GRID ? sms : MAX_GRID;
+  f->s.smem_max = smem;
+  f->s.slots = c->a.scratch;
+  f->s.counters = (int *)((char *)c->a.scratch + slots_bytes());
+  if (cudaMemsetAsync(f->s.counters, 0, MAX_TILES * sizeof(int), c->stream) != cudaSuccess ||
+      cudaFuncSetAttribute(gemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) {
+    delete f;
+    c->err = "tensor-core GEMM set-up failed";
+    return OURO_ECUDA;
+  }
+  for (int w = 0; w < 2; ++w) {
+    ModelRt &M = c->m[w];
+    if (!M.present || !shape_ok(M.d)) continue;
+    const ouro_model_desc &d = M.d;
+    FastModel &fm = f->s.m[w];
+    const int dq = d.n_heads * d.head_dim, dkv = d.n_kv_heads * d.head_dim;
+    bool ok = true;
+    fm.layers.resize(d.n_layers);
+    for (int l = 0; l < d.n_layers && ok; ++l) {
+      LayerMaps &lm = fm.layers[l];
+      ok = make_map(&lm.wq, M.wq[l], dq, d.d_model, TILE_N) && make_map(&lm.wk, M.wk[l], dkv, d.d_model, TILE_N) &&
+           make_map(&lm.wv, M.wv[l], dkv, d.d_model, TILE_N) && make_map(&lm.wo, M.wo[l], d.d_model, dq, TILE_N) &&
+           make_map(&lm.wg, M.w_gate[l], d.d_ffn, d.d_model, 64) && make_map(&lm.wu, M.w_up[l], d.d_ffn, d.d_model, 64) &&
+           make_map(&lm.wd, M.w_down[l], d.d_model, d.d_ffn, TILE_N);
+    }
+    ok = ok && make_map(&fm.head, M.lm_head, d.vocab, d.d_model, TILE_N) &&
+         make_map(&fm.x_d, c->a.xn, OURO_MAX_ROWS, d.d_model, 16) && make_map(&fm.x_q, c->a.att, OURO_MAX_ROWS, dq, 16) &&
+         make_map(&fm.x_f, c->a.act, OURO_MAX_ROWS, d.d_ffn, 16);
+    if (!ok) {
+      delete f;
+      c->err = "cuTensorMapEncodeTiled failed";
+      return OURO_ECUDA;
+    }
+    fm.ok = true;
+  }
+  c->fast = f;
+  return OURO_OK;
+}
+
+void ouro_fast_teardown(ouro_ctx *c) {
+  delete c->fast;
+  c->fast = nullptr;
+}
+
+static void launch_gemm_tc(ouro_ctx *c, GemmParams &p, int K, int rows) {
+  OURO_COUNT_LAUNCH();
+  FastState &s = c->fast->s;
+  p.kb = K / BLOCK_K;
+  p.rows = rows;
+  p.t_pad = (rows + 15) & ~15;
+  p.stages = stages_for(p.t_pad, s.smem_max);
+  p.scratch = s.slots;
+  p.counters = s.counters;
+  p.status = &c->st->status;
+  int total = p.tiles * p.kb;
+  int grid = total < s.grid ? total : s.grid;
+  gemm_tc_kernel<<<grid, THREADS, s.smem_max, c->stream>>>(p);
+}
+
+// One decoder layer with the tensor-core GEMMs; OURO_ESTATE when the model does not qualify.
+int ouro_fast_layer(ouro_ctx *c, int which, int l, int rows) {
+  if (!c->fast || !c->fast->s.m[which].ok) return OURO_ESTATE;
+  ModelRt &M = c->m[which];
+  FastModel &fm = c->fast->s.m[which];
+  const ouro_model_desc &d = M.d;
+  const int dq = d.n_heads * d.head_dim, dkv = d.n_kv_heads * d.head_dim;
+  Activations &a = c->a;
+  cudaStream_t s = c->stream;
+  LayerMaps &lm = fm.layers[l];
+  auto tiles = [](int n) { return (n + TILE_N - 1) / TILE_N; };
+  { ProfScope ps(c, OURO_PROF_NORM); launch_rmsnorm(OURO_BF16, a.x, M.attn_norm[l], rows, d.d_model, d.rms_eps, a.xn, s); }
+  {
+    ProfScope ps(c, OURO_PROF_QKV);
+    GemmParams p{};
+    p.a[0] = lm.wq; p.a[1] = lm.wk; p.a[2] = lm.wv;
+    p.a_tiles[0] = tiles(dq); p.a_tiles[1] = tiles(dkv); p.a_tiles[2] = tiles(dkv);
+    p.a_rows[0] = dq; p.a_rows[1] = dkv; p.a_rows[2] = dkv;
+    p.a_count = 3;
+    p.b = fm.x_d;
+    p.mode = MODE_STORE;
+    p.tiles = p.a_tiles[0] + p.a_tiles[1] + p.a_tiles[2];
+    p.out_f32 = a.qkv;
+    p.ldo = dq + 2 * dkv;
+    launch_gemm_tc(c, p, d.d_model, rows);
+  }
+  { ProfScope ps(c, OURO_PROF_ROPE); launch_rope_append(d, a.qkv, M.blk.pos, M.rope_cos, M.rope_sin, rows, M.L, l, a.q, M.k_cache, M.v_cache, s); }
+  { ProfScope ps(c, OURO_PROF_ATTENTION); launch_attention_simple(d, a.q, M.k_cache, M.v_cache, M.blk, rows, l, a.att, s); }
+  {
+    ProfScope ps(c, OURO_PROF_WO);
+    GemmParams p{};
+    p.a[0] = lm.wo; p.a_tiles[0] = tiles(d.d_model); p.a_rows[0] = d.d_model; p.a_count = 1;
+    p.b = fm.x_q;
+    p.mode = MODE_RESIDUAL;
+    p.tiles = p.a_tiles[0];
+    p.out_f32 = a.x;
+    p.ldo = d.d_model;
+    launch_gemm_tc(c, p, dq, rows);
+  }
+  { ProfScope ps(c, OURO_PROF_NORM); launch_rmsnorm(OURO_BF16, a.x, M.ffn_norm[l], rows, d.d_model, d.rms_eps, a.xn, s); }
+  {
+    ProfScope ps(c, OURO_PROF_GATEUP);
+    GemmParams p{};
+    p.a[0] = lm.wg; p.a[1] = lm.wu; p.a_rows[0] = d.d_ffn; p.a_count = 2;
+    p.b = fm.x_d;
+    p.mode = MODE_SWIGLU;
+    p.tiles = (d.d_ffn + 63) / 64;
+    p.out_bf16 = (__nv_bfloat16 *)a.act;
+    launch_gemm_tc(c, p, d.d_model, rows);
+  }
+  {
+    ProfScope ps(c, OURO_PROF_DOWN);
+    GemmParams p{};
+    p.a[0] = lm.wd; p.a_tiles[0] = tiles(d.d_model); p.a_rows[0] = d.d_model; p.a_count = 1;
+    p.b = fm.x_f;
+    p.mode = MODE_RESIDUAL;
+    p.tiles = p.a_tiles[0];
+    p.out_f32 = a.x;
+    p.ldo = d.d_model;
+    launch_gemm_tc(c, p, d.d_ffn, rows);
+  }
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) {
+    c->err = std::string("tensor-core layer launch: ") + cudaGetErrorString(e);
+    return OURO_ECUDA;
+  }
+  return OURO_OK;
+}
+
+int ouro_fast_head(ouro_ctx *c, int which, int rows, float *logits) {
+  if (!c->fast || !c->fast->s.m[which].ok) return OURO_ESTATE;
+  ModelRt &M = c->m[which];
+  FastModel &fm = c->fast->s.m[which];
+  const ouro_model_desc &d = M.d;
+  { ProfScope ps(c, OURO_PROF_NORM); launch_rmsnorm(OURO_BF16, c->a.x, M.final_norm, rows, d.d_model, d.rms_eps, c->a.xn, c->stream); }
+  ProfScope ps(c, OURO_PROF_HEAD);
+  GemmParams p{};
+  p.a[0] = fm.head; p.a_tiles[0] = (d.vocab + TILE_N - 1) / TILE_N; p.a_rows[0] = d.vocab; p.a_count = 1;
+  p.b = fm.x_d;
+  p.mode = MODE_STORE;
+  p.tiles = p.a_tiles[0];
+  p.out_f32 = logits;
+  p.ldo = d.vocab;
+  launch_gemm_tc(c, p, d.d_model, rows);
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) {
+    c->err = std::string("tensor-core head launch: ") + cudaGetErrorString(e);
+    return OURO_ECUDA;
+  }
+  return OURO_OK;
+}

@@ -74,7 +74,10 @@ struct Activations {  // sized for OURO_MAX_ROWS rows of the larger model
   size_t scratch_bytes;
 };
 
+struct ouro_fast;   // tensor maps and launch state of the tensor-core paths (gemm_tc.cu)
+
 struct ouro_ctx {
+  ouro_fast *fast = nullptr;
   ModelRt m[2];
   ouro_params p{};
   cudaStream_t stream = nullptr;
@@ -101,6 +104,7 @@ struct ouro_ctx {
   double prof_ms = 0.0;
   long prof_launches = 0;
 };
+void ouro_fast_teardown(ouro_ctx *c);
 void prof_mark(ouro_ctx *c, int kernel_class);   // call before and after the launches of a class
 struct ProfScope {
   ouro_ctx *c; int k;

@@ -479,3 +479,42 @@ def test_edge_cases():
     t2, p2, g2, vis = ob.build_block(19, prompt[-1], d, cands)
     assert np.abs(logits.cpu().numpy() - tf.forward(W2, cache, t2, p2, vis)).max() < FP32_TOL
     eng.close(); e2.close()
+
+
+# ----------------------------------------------- full-size verify step (the benchmark's configuration)
+
+@pytest.mark.parametrize("L", [1024, 4096])
+def test_verify_step_full_size_c2(L):
+    """One 7B-shaped layer + LM head, 37-row candidate block on a random KV cache of L tokens, exactly as
+    bench.py runs it: logits of every row against the oracle, acceptance and pool bit exact."""
+    T, _, P, _ = synth.config("C2")
+    w = synth.model_weights(T, 0, device="cuda:0")
+    eng = binding.Engine(T, w, P)
+    k, v = synth.kv_fill(T, 1, L, device="cuda:0")
+    eng.tm.k_cache.copy_(k); eng.tm.v_cache.copy_(v)
+    W = tf.Weights(T, {n: (t.cpu() if n != "layers" else [{a: b.cpu() for a, b in lw.items()} for lw in t]) for n, t in w.items()})
+    cache = tf.KVCache(T, k.double().cpu().numpy(), v.double().cpu().numpy(), L)
+    rng = np.random.default_rng(L)
+    d = rng.integers(0, T.vocab, P.gamma).tolist()
+    grams = np.concatenate([np.full((P.K, 1), d[-1]), rng.integers(0, T.vocab, (P.K, P.S))], axis=1)
+    eng.phrase_update(grams)
+    pool = oracle_pool(P)
+    for g in grams:
+        pool.insert(g)
+    eng.set_state(L, 17)
+    eng.assemble_candidates(draft=d)
+    tok = eng.block_get()[0].tolist()
+    tokens, pos, group, vis = ob.build_block(L, 17, d, pool.lookup(d[-1], P.K))
+    assert tok == tokens and len(tok) == 37
+    am, logits = eng.verify_forward(want_logits=True)
+    want = tf.forward(W, cache, tokens, pos, vis)
+    got = logits[:37].cpu().numpy().astype(np.float64)
+    _bf16_tol(got, want)
+    o = am[:37].cpu().numpy().tolist()
+    n, chosen, A, acc = eng.accept_and_compact()
+    A2, j2, m2, acc2 = ob.accept(tokens, o, P.gamma, P.S, P.K)
+    assert (n, chosen, A, acc.tolist()) == (len(acc2), j2, A2, acc2)
+    seq = [0] * L + [17] + acc2
+    pool.apply(ob.harvest_ops(tokens, o, P.gamma, P.S, P.K, A2, seq, len(acc2), P))
+    assert gpu_pool_rows(eng) == pool_rows(pool)
+    eng.close()
