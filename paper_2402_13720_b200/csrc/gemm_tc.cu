@@ -121,30 +121,48 @@ __device__ __forceinline__ void fence_before_sync() { asm volatile("tcgen05.fenc
 __device__ __forceinline__ void fence_after_sync() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void epi_barrier() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
 
-struct Span {  // one piece of this CTA's iteration range: k-blocks [kb0, kb1) of `tile`
-  int tile, kb0, kb1, n_contrib, slot;
+struct Span {  // one piece of this CTA's work: k-blocks [kb0, kb1) of `tile`
+  int tile, kb0, kb1, n_contrib, slot, first_owner;
 };
 
-// Walks the CTA's contiguous share of the (tile, k-block) space; identical in every warp role.
+// Work of one CTA, identical in every warp role.  The last R = tiles mod grid tiles are cut stream-K
+// fashion into equal contiguous spans of the (tile, k-block) space and come first, so that their partial
+// sums are added up while the whole tiles (tile c, c + grid, ...) that follow are still streaming.
 struct SpanWalker {
-  int it, end, kb, per;
+  int kb, per, t0, it, end, whole;
   __device__ SpanWalker(const GemmParams &p) {
-    int total = p.tiles * p.kb;
+    kb = p.kb;
+    t0 = (p.tiles / (int)gridDim.x) * (int)gridDim.x;      // tiles [0, t0) are handled whole
+    int total = (p.tiles - t0) * kb;
     per = (total + gridDim.x - 1) / gridDim.x;
     it = min(total, (int)blockIdx.x * per);
     end = min(total, it + per);
-    kb = p.kb;
+    whole = blockIdx.x;
   }
+  __device__ int owner_slot(int tile, int owner) const { return ((tile - t0) * kb <= owner * per) ? 0 : 1; }
   __device__ bool next(Span &s) {
-    if (it >= end) return false;
-    s.tile = it / kb;
-    s.kb0 = it - s.tile * kb;
-    s.kb1 = min(kb, s.kb0 + (end - it));
-    int first_owner = (s.tile * kb) / per, last_owner = (s.tile * kb + kb - 1) / per;
-    s.n_contrib = last_owner - first_owner + 1;
-    s.slot = (s.tile * kb <= (int)blockIdx.x * per) ? 0 : 1;   // first or last piece of this CTA
-    it += s.kb1 - s.kb0;
-    return true;
+    if (it < end) {
+      int rel = it / kb;
+      s.tile = t0 + rel;
+      s.kb0 = it - rel * kb;
+      s.kb1 = min(kb, s.kb0 + (end - it));
+      s.first_owner = (rel * kb) / per;
+      s.n_contrib = (rel * kb + kb - 1) / per - s.first_owner + 1;
+      s.slot = owner_slot(s.tile, blockIdx.x);               // first or last piece of this CTA
+      it += s.kb1 - s.kb0;
+      return true;
+    }
+    if (whole < t0) {
+      s.tile = whole;
+      s.kb0 = 0;
+      s.kb1 = kb;
+      s.n_contrib = 1;
+      s.slot = 0;
+      s.first_owner = blockIdx.x;
+      whole += gridDim.x;
+      return true;
+    }
+    return false;
   }
 };
 
@@ -352,34 +370,87 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_tc_kernel(const __grid_consta
         epi_barrier();
         if (last) {
           __threadfence();
-          const int per = w.per;
-          const int first_owner = (s.tile * p.kb) / per;
+          // Sum the partial tiles in ascending K order.  Everything one thread needs for a batch of tokens
+          // is requested before the first add, so the pass runs at L2 bandwidth rather than L2 latency.
           if (p.mode == MODE_SWIGLU) {
             const int F = p.a_rows[0];
-            // 128 threads: thread -> (feature r = et & 63, token parity et >> 6)
-            const int r = et & 63, feat = s.tile * 64 + r;
-            for (int t = et >> 6; t < p.rows; t += 2) {
-              float g = 0.f, u = 0.f;
-              for (int c = 0; c < s.n_contrib; ++c) {
-                int owner = first_owner + c;
-                int slot = (s.tile * p.kb <= owner * per) ? 0 : 1;
-                const float *src = p.scratch + ((size_t)owner * 2 + slot) * SLOT_FLOATS + (size_t)t * TILE_N;
-                g += __ldcg(src + r);
-                u += __ldcg(src + 64 + r);
+            const int ng = et & 15, tg = et >> 4;                     // 4 features x tokens tg, tg+8, ..
+            const int feat = s.tile * 64 + 4 * ng;
+            for (int tb = 0; tb < p.rows; tb += 32) {
+              float4 g[4], u[4];
+#pragma unroll
+              for (int j = 0; j < 4; ++j) g[j] = u[j] = make_float4(0.f, 0.f, 0.f, 0.f);
+              for (int c0 = 0; c0 < s.n_contrib; c0 += 4) {
+                float4 tg4[4][4], tu4[4][4];
+#pragma unroll
+                for (int cc = 0; cc < 4; ++cc) {
+                  int owner = s.first_owner + c0 + cc;
+                  const float *src = p.scratch + ((size_t)owner * 2 + w.owner_slot(s.tile, owner)) * SLOT_FLOATS + 4 * ng;
+#pragma unroll
+                  for (int j = 0; j < 4; ++j) {
+                    int t = tb + tg + 8 * j;
+                    bool in = c0 + cc < s.n_contrib && t < p.rows;
+                    tg4[cc][j] = in ? __ldcg((const float4 *)(src + (size_t)t * TILE_N)) : make_float4(0.f, 0.f, 0.f, 0.f);
+                    tu4[cc][j] = in ? __ldcg((const float4 *)(src + (size_t)t * TILE_N + 64)) : make_float4(0.f, 0.f, 0.f, 0.f);
+                  }
+                }
+#pragma unroll
+                for (int cc = 0; cc < 4; ++cc)
+#pragma unroll
+                  for (int j = 0; j < 4; ++j) {
+                    g[j].x += tg4[cc][j].x; g[j].y += tg4[cc][j].y; g[j].z += tg4[cc][j].z; g[j].w += tg4[cc][j].w;
+                    u[j].x += tu4[cc][j].x; u[j].y += tu4[cc][j].y; u[j].z += tu4[cc][j].z; u[j].w += tu4[cc][j].w;
+                  }
               }
-              if (feat < F) p.out_bf16[(size_t)t * F + feat] = __float2bfloat16_rn(g / (1.0f + __expf(-g)) * u);
+#pragma unroll
+              for (int j = 0; j < 4; ++j) {
+                int t = tb + tg + 8 * j;
+                if (t < p.rows && feat < F) {
+                  __nv_bfloat162 lo = __floats2bfloat162_rn(g[j].x / (1.0f + __expf(-g[j].x)) * u[j].x,
+                                                            g[j].y / (1.0f + __expf(-g[j].y)) * u[j].y);
+                  __nv_bfloat162 hi = __floats2bfloat162_rn(g[j].z / (1.0f + __expf(-g[j].z)) * u[j].z,
+                                                            g[j].w / (1.0f + __expf(-g[j].w)) * u[j].w);
+                  uint2 pk = make_uint2(*(uint32_t *)&lo, *(uint32_t *)&hi);
+                  *(uint2 *)(p.out_bf16 + (size_t)t * F + feat) = pk;
+                }
+              }
             }
           } else {
-            for (int t = 0; t < p.rows; ++t) {
-              float acc = 0.f;
-              for (int c = 0; c < s.n_contrib; ++c) {
-                int owner = first_owner + c;
-                int slot = (s.tile * p.kb <= owner * per) ? 0 : 1;
-                acc += __ldcg(p.scratch + ((size_t)owner * 2 + slot) * SLOT_FLOATS + (size_t)t * TILE_N + nl);
+            const int ng = et & 31, tg = et >> 5;                     // 4 columns x tokens tg, tg+4, ..
+            for (int tb = 0; tb < p.rows; tb += 32) {
+              float4 acc[8];
+#pragma unroll
+              for (int j = 0; j < 8; ++j) acc[j] = make_float4(0.f, 0.f, 0.f, 0.f);
+              for (int c0 = 0; c0 < s.n_contrib; c0 += 4) {
+                float4 tmp[4][8];
+#pragma unroll
+                for (int cc = 0; cc < 4; ++cc) {
+                  int owner = s.first_owner + c0 + cc;
+                  const float *src = p.scratch + ((size_t)owner * 2 + w.owner_slot(s.tile, owner)) * SLOT_FLOATS + 4 * ng;
+#pragma unroll
+                  for (int j = 0; j < 8; ++j) {
+                    int t = tb + tg + 4 * j;
+                    tmp[cc][j] = (c0 + cc < s.n_contrib && t < p.rows) ? __ldcg((const float4 *)(src + (size_t)t * TILE_N))
+                                                                       : make_float4(0.f, 0.f, 0.f, 0.f);
+                  }
+                }
+#pragma unroll
+                for (int cc = 0; cc < 4; ++cc)
+#pragma unroll
+                  for (int j = 0; j < 8; ++j) {
+                    acc[j].x += tmp[cc][j].x; acc[j].y += tmp[cc][j].y; acc[j].z += tmp[cc][j].z; acc[j].w += tmp[cc][j].w;
+                  }
               }
-              if (nl < valid) {
-                float *y = p.out_f32 + (size_t)t * p.ldo + col0 + nl;
-                *y = p.mode == MODE_RESIDUAL ? *y + acc : acc;
+              const int col = col0 + 4 * ng;
+#pragma unroll
+              for (int j = 0; j < 8; ++j) {
+                int t = tb + tg + 4 * j;
+                if (t >= p.rows) continue;
+                float *y = p.out_f32 + (size_t)t * p.ldo + col;
+                float vals[4] = {acc[j].x, acc[j].y, acc[j].z, acc[j].w};
+#pragma unroll
+                for (int e = 0; e < 4; ++e)
+                  if (4 * ng + e < valid) y[e] = p.mode == MODE_RESIDUAL ? y[e] + vals[e] : vals[e];
               }
             }
           }
