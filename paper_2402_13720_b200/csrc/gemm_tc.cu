@@ -499,6 +499,7 @@ struct FastState {
   int smem_max = 0;
   float *slots = nullptr;
   int *counters = nullptr;
+  float *attn_part = nullptr;   // per-chunk softmax pieces of the split attention
 };
 constexpr int MAX_TILES = 4096;
 
@@ -515,8 +516,10 @@ int stages_for(int t_pad, int smem_max) {
 
 struct ouro_fast { FastState s; };
 
-size_t ouro_scratch_bytes(const ouro_model_desc *, const ouro_model_desc *) {
-  return slots_bytes() + MAX_TILES * sizeof(int) + 256;
+size_t ouro_scratch_bytes(const ouro_model_desc *t, const ouro_model_desc *d) {
+  size_t attn = attention_tc_scratch_bytes(*t);
+  if (d && attention_tc_scratch_bytes(*d) > attn) attn = attention_tc_scratch_bytes(*d);
+  return slots_bytes() + MAX_TILES * sizeof(int) + 256 + attn;
 }
 
 static bool shape_ok(const ouro_model_desc &d) {
@@ -550,8 +553,10 @@ int ouro_fast_setup(ouro_ctx *c) {
   f->s.smem_max = smem;
   f->s.slots = c->a.scratch;
   f->s.counters = (int *)((char *)c->a.scratch + slots_bytes());
+  f->s.attn_part = (float *)((char *)c->a.scratch + slots_bytes() + MAX_TILES * sizeof(int) + 256);
   if (cudaMemsetAsync(f->s.counters, 0, MAX_TILES * sizeof(int), c->stream) != cudaSuccess ||
-      cudaFuncSetAttribute(gemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) {
+      cudaFuncSetAttribute(gemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess ||
+      attention_tc_setup() != OURO_OK) {
     delete f;
     c->err = "tensor-core GEMM set-up failed";
     return OURO_ECUDA;
@@ -632,7 +637,13 @@ int ouro_fast_layer(ouro_ctx *c, int which, int l, int rows) {
     launch_gemm_tc(c, p, d.d_model, rows);
   }
   { ProfScope ps(c, OURO_PROF_ROPE); launch_rope_append(d, a.qkv, M.blk.pos, M.rope_cos, M.rope_sin, rows, M.L, l, a.q, M.k_cache, M.v_cache, s); }
-  { ProfScope ps(c, OURO_PROF_ATTENTION); launch_attention_simple(d, a.q, M.k_cache, M.v_cache, M.blk, rows, l, a.att, s); }
+  {
+    ProfScope ps(c, OURO_PROF_ATTENTION);
+    if (attention_tc_supported(d))
+      launch_attention_tc(d, a.q, M.k_cache, M.v_cache, M.blk, rows, M.L, M.L + rows, l, c->fast->s.attn_part, a.att, s);
+    else
+      launch_attention_simple(d, a.q, M.k_cache, M.v_cache, M.blk, rows, l, a.att, s);
+  }
   {
     ProfScope ps(c, OURO_PROF_WO);
     GemmParams p{};

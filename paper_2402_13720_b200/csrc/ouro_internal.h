@@ -152,3 +152,10 @@ void launch_rope_append(const ouro_model_desc &d, const float *qkv, const int32_
                         cudaStream_t s);
 void launch_attention_simple(const ouro_model_desc &d, const void *q, const void *k_cache, const void *v_cache,
                              const BlockDev &b, int rows, int layer, void *out, cudaStream_t s);
+
+// ---- attn_tc.cu --------------------------------------------------------------------------------
+bool attention_tc_supported(const ouro_model_desc &d);
+size_t attention_tc_scratch_bytes(const ouro_model_desc &d);
+int attention_tc_setup();
+void launch_attention_tc(const ouro_model_desc &d, const void *q, const void *k_cache, const void *v_cache, const BlockDev &b,
+                         int rows, int L, int n_vis_max, int layer, float *part, void *out, cudaStream_t s);
