@@ -371,7 +371,7 @@ extern "C" int ouro_profile_read(ouro_ctx *c, float *ms_total, int32_t *launches
 
 // ----------------------------------------------------------------------------------- forward
 int ouro_fast_layer(ouro_ctx *c, int which, int layer, int rows);          // tensor-core layer; OURO_ESTATE = not available
-int ouro_fast_head(ouro_ctx *c, int which, int rows, float *logits);      // tensor-core LM head
+int ouro_fast_head(ouro_ctx *c, int which, int rows, float *logits, int32_t *argmax_dev);   // tensor-core LM head + argmax
 
 static int forward(ouro_ctx *c, int which, int32_t *argmax_dev, float *logits_dev) {
   ModelRt &M = c->m[which];
@@ -409,18 +409,20 @@ static int forward(ouro_ctx *c, int which, int32_t *argmax_dev, float *logits_de
       launch_gemm_simple(dt, a.act, wd, rows, d.d_ffn, a.x, d.d_model, EPI_RESIDUAL, s);
     }
   }
-  float *logits = logits_dev ? logits_dev : a.logits;
-  int rc = ouro_fast_head(c, which, rows, logits);
+  int rc = ouro_fast_head(c, which, rows, logits_dev, argmax_dev);
   if (rc == OURO_ESTATE) {
+    float *logits = logits_dev ? logits_dev : a.logits;
     { ProfScope ps(c, OURO_PROF_NORM); launch_rmsnorm(dt, a.x, M.final_norm, rows, d.d_model, d.rms_eps, a.xn, s); }
-    ProfScope ps(c, OURO_PROF_HEAD);
-    GemmSegs head{{M.lm_head, nullptr, nullptr}, {d.vocab, 0, 0}, 1};
-    launch_gemm_simple(dt, a.xn, head, rows, d.d_model, logits, d.vocab, EPI_STORE, s);
+    {
+      ProfScope ps(c, OURO_PROF_HEAD);
+      GemmSegs head{{M.lm_head, nullptr, nullptr}, {d.vocab, 0, 0}, 1};
+      launch_gemm_simple(dt, a.xn, head, rows, d.d_model, logits, d.vocab, EPI_STORE, s);
+    }
+    ProfScope pa(c, OURO_PROF_ARGMAX);
+    launch_argmax(logits, rows, d.vocab, argmax_dev, s);
   } else if (rc != OURO_OK) {
     return rc;
   }
-  ProfScope pa(c, OURO_PROF_ARGMAX);
-  launch_argmax(logits, rows, d.vocab, argmax_dev, s);
   CKL();
   return OURO_OK;
 }

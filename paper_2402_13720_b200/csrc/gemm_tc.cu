@@ -33,7 +33,7 @@ constexpr uint32_t SPIN_LIMIT = 1u << 24;
 constexpr unsigned long long HINT_EVICT_FIRST = 0x12F0000000000000ull;
 constexpr unsigned long long HINT_EVICT_LAST = 0x14F0000000000000ull;
 
-enum { MODE_STORE = 0, MODE_RESIDUAL = 1, MODE_SWIGLU = 2 };
+enum { MODE_STORE = 0, MODE_RESIDUAL = 1, MODE_SWIGLU = 2, MODE_HEAD = 3 };   // HEAD: per-tile row maxima (+ optional logits)
 
 struct GemmParams {
   CUtensorMap a[3];   // weight matrices stacked along the output dimension (q|k|v), or gate and up
@@ -50,6 +50,8 @@ struct GemmParams {
   float *out_f32;     // MODE_STORE / MODE_RESIDUAL: [rows, ldo]
   int ldo;
   __nv_bfloat16 *out_bf16;  // MODE_SWIGLU: [rows, F]
+  float *tile_max;    // MODE_HEAD: [tiles][128] largest logit of each token inside the tile ...
+  int *tile_arg;      //            ... and its vocabulary index (smallest index among equals)
   float *scratch;     // [grid][2][t][128] partial tiles
   int *counters;      // [tiles], zero between launches
   int *status;        // context status word
@@ -183,7 +185,7 @@ __device__ __forceinline__ void locate(const GemmParams &p, int tile, int &seg, 
 
 // Final values of one output row n (this thread) for tokens t0..t0+15.
 __device__ __forceinline__ void store_chunk(const GemmParams &p, int col, bool n_ok, int t0, const float *v) {
-  if (!n_ok) return;
+  if (!n_ok || !p.out_f32) return;
 #pragma unroll
   for (int i = 0; i < 16; ++i) {
     int t = t0 + i;
@@ -338,9 +340,41 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_tc_kernel(const __grid_consta
             epi_barrier();
           }
         } else {
+          float *xv = xchg;                                   // [4 quarters][128 tokens] best value
+          int *xi = (int *)(xchg + 4 * OURO_MAX_ROWS);        //                         and its index
           for (int t0 = 0; t0 < p.t_pad; t0 += 16) {
             tmem_ld16(taddr + t0, v);
             store_chunk(p, col0 + nl, nl < valid, t0, v);
+            if (p.mode == MODE_HEAD) {
+#pragma unroll
+              for (int i = 0; i < 16; ++i) {
+                float bv = nl < valid ? v[i] : -INFINITY;
+                int bi = col0 + nl;
+#pragma unroll
+                for (int o = 16; o; o >>= 1) {
+                  float ov = __shfl_xor_sync(0xffffffffu, bv, o);
+                  int oi = __shfl_xor_sync(0xffffffffu, bi, o);
+                  if (ov > bv || (ov == bv && oi < bi)) { bv = ov; bi = oi; }
+                }
+                if (lane == 0) { xv[q * OURO_MAX_ROWS + t0 + i] = bv; xi[q * OURO_MAX_ROWS + t0 + i] = bi; }
+              }
+            }
+          }
+          if (p.mode == MODE_HEAD) {
+            epi_barrier();
+            if (et < p.rows) {
+              float bv = xv[et];
+              int bi = xi[et];
+#pragma unroll
+              for (int qq = 1; qq < 4; ++qq) {
+                float ov = xv[qq * OURO_MAX_ROWS + et];
+                int oi = xi[qq * OURO_MAX_ROWS + et];
+                if (ov > bv || (ov == bv && oi < bi)) { bv = ov; bi = oi; }
+              }
+              p.tile_max[(size_t)s.tile * OURO_MAX_ROWS + et] = bv;
+              p.tile_arg[(size_t)s.tile * OURO_MAX_ROWS + et] = bi;
+            }
+            epi_barrier();
           }
         }
         fence_before_sync();
@@ -442,10 +476,32 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_tc_kernel(const __grid_consta
                   }
               }
               const int col = col0 + 4 * ng;
+              if (p.mode == MODE_HEAD) {
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {            // the 32 lanes of this warp cover the tile's 128 columns
+                  int t = tb + tg + 4 * j;
+                  float vals[4] = {acc[j].x, acc[j].y, acc[j].z, acc[j].w};
+                  float bv = -INFINITY;
+                  int bi = col;
+#pragma unroll
+                  for (int e = 0; e < 4; ++e)
+                    if (4 * ng + e < valid && vals[e] > bv) { bv = vals[e]; bi = col + e; }
+#pragma unroll
+                  for (int o = 16; o; o >>= 1) {
+                    float ov = __shfl_xor_sync(0xffffffffu, bv, o);
+                    int oi = __shfl_xor_sync(0xffffffffu, bi, o);
+                    if (ov > bv || (ov == bv && oi < bi)) { bv = ov; bi = oi; }
+                  }
+                  if (lane == 0 && t < p.rows) {
+                    p.tile_max[(size_t)s.tile * OURO_MAX_ROWS + t] = bv;
+                    p.tile_arg[(size_t)s.tile * OURO_MAX_ROWS + t] = bi;
+                  }
+                }
+              }
 #pragma unroll
               for (int j = 0; j < 8; ++j) {
                 int t = tb + tg + 4 * j;
-                if (t >= p.rows) continue;
+                if (t >= p.rows || !p.out_f32) continue;
                 float *y = p.out_f32 + (size_t)t * p.ldo + col;
                 float vals[4] = {acc[j].x, acc[j].y, acc[j].z, acc[j].w};
 #pragma unroll
@@ -500,10 +556,13 @@ struct FastState {
   float *slots = nullptr;
   int *counters = nullptr;
   float *attn_part = nullptr;   // per-chunk softmax pieces of the split attention
+  float *tile_max = nullptr;    // LM head: per-tile best logit and index of every token
+  int *tile_arg = nullptr;
 };
 constexpr int MAX_TILES = 4096;
 
 size_t slots_bytes() { return (size_t)MAX_GRID * 2 * SLOT_FLOATS * sizeof(float); }
+size_t tile_best_bytes() { return (size_t)MAX_TILES * OURO_MAX_ROWS * 4; }
 
 int stages_for(int t_pad, int smem_max) {
   int stage = A_BYTES + t_pad * BLOCK_K * 2;
@@ -519,7 +578,7 @@ struct ouro_fast { FastState s; };
 size_t ouro_scratch_bytes(const ouro_model_desc *t, const ouro_model_desc *d) {
   size_t attn = attention_tc_scratch_bytes(*t);
   if (d && attention_tc_scratch_bytes(*d) > attn) attn = attention_tc_scratch_bytes(*d);
-  return slots_bytes() + MAX_TILES * sizeof(int) + 256 + attn;
+  return slots_bytes() + MAX_TILES * sizeof(int) + 256 + 2 * tile_best_bytes() + attn;
 }
 
 static bool shape_ok(const ouro_model_desc &d) {
@@ -553,7 +612,9 @@ int ouro_fast_setup(ouro_ctx *c) {
   f->s.smem_max = smem;
   f->s.slots = c->a.scratch;
   f->s.counters = (int *)((char *)c->a.scratch + slots_bytes());
-  f->s.attn_part = (float *)((char *)c->a.scratch + slots_bytes() + MAX_TILES * sizeof(int) + 256);
+  f->s.tile_max = (float *)((char *)c->a.scratch + slots_bytes() + MAX_TILES * sizeof(int) + 256);
+  f->s.tile_arg = (int *)((char *)f->s.tile_max + tile_best_bytes());
+  f->s.attn_part = (float *)((char *)f->s.tile_arg + tile_best_bytes());
   if (cudaMemsetAsync(f->s.counters, 0, MAX_TILES * sizeof(int), c->stream) != cudaSuccess ||
       cudaFuncSetAttribute(gemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess ||
       attention_tc_setup() != OURO_OK) {
@@ -685,21 +746,58 @@ int ouro_fast_layer(ouro_ctx *c, int which, int l, int rows) {
   return OURO_OK;
 }
 
-int ouro_fast_head(ouro_ctx *c, int which, int rows, float *logits) {
+// Final norm, LM head and greedy choice.  The GEMM's epilogue keeps, per 128-entry vocabulary tile, each
+// token's best logit and index; a small kernel then picks the best tile per token.  logits may be NULL.
+__global__ void argmax_tiles_kernel(const float *tile_max, const int *tile_arg, int tiles, int32_t *out) {
+  const int t = blockIdx.x;
+  float bv = -INFINITY;
+  int bi = INT_MAX;
+  for (int i = threadIdx.x; i < tiles; i += blockDim.x) {
+    float v = tile_max[(size_t)i * OURO_MAX_ROWS + t];
+    int a = tile_arg[(size_t)i * OURO_MAX_ROWS + t];
+    if (v > bv || (v == bv && a < bi)) { bv = v; bi = a; }
+  }
+  __shared__ float sv[8];
+  __shared__ int si[8];
+#pragma unroll
+  for (int o = 16; o; o >>= 1) {
+    float ov = __shfl_xor_sync(0xffffffffu, bv, o);
+    int oi = __shfl_xor_sync(0xffffffffu, bi, o);
+    if (ov > bv || (ov == bv && oi < bi)) { bv = ov; bi = oi; }
+  }
+  if ((threadIdx.x & 31) == 0) { sv[threadIdx.x >> 5] = bv; si[threadIdx.x >> 5] = bi; }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    for (int w = 1; w < (int)(blockDim.x >> 5); ++w)
+      if (sv[w] > bv || (sv[w] == bv && si[w] < bi)) { bv = sv[w]; bi = si[w]; }
+    out[t] = bi == INT_MAX ? 0 : bi;
+  }
+}
+
+int ouro_fast_head(ouro_ctx *c, int which, int rows, float *logits, int32_t *argmax_dev) {
   if (!c->fast || !c->fast->s.m[which].ok) return OURO_ESTATE;
   ModelRt &M = c->m[which];
   FastModel &fm = c->fast->s.m[which];
   const ouro_model_desc &d = M.d;
   { ProfScope ps(c, OURO_PROF_NORM); launch_rmsnorm(OURO_BF16, c->a.x, M.final_norm, rows, d.d_model, d.rms_eps, c->a.xn, c->stream); }
-  ProfScope ps(c, OURO_PROF_HEAD);
-  GemmParams p{};
-  p.a[0] = fm.head; p.a_tiles[0] = (d.vocab + TILE_N - 1) / TILE_N; p.a_rows[0] = d.vocab; p.a_count = 1;
-  p.b = fm.x_d;
-  p.mode = MODE_STORE;
-  p.tiles = p.a_tiles[0];
-  p.out_f32 = logits;
-  p.ldo = d.vocab;
-  launch_gemm_tc(c, p, d.d_model, rows);
+  {
+    ProfScope ps(c, OURO_PROF_HEAD);
+    GemmParams p{};
+    p.a[0] = fm.head; p.a_tiles[0] = (d.vocab + TILE_N - 1) / TILE_N; p.a_rows[0] = d.vocab; p.a_count = 1;
+    p.b = fm.x_d;
+    p.mode = MODE_HEAD;
+    p.tiles = p.a_tiles[0];
+    p.out_f32 = logits;
+    p.ldo = d.vocab;
+    p.tile_max = c->fast->s.tile_max;
+    p.tile_arg = c->fast->s.tile_arg;
+    launch_gemm_tc(c, p, d.d_model, rows);
+  }
+  {
+    ProfScope ps(c, OURO_PROF_ARGMAX);
+    OURO_COUNT_LAUNCH();
+    argmax_tiles_kernel<<<rows, 128, 0, c->stream>>>(c->fast->s.tile_max, c->fast->s.tile_arg, (d.vocab + TILE_N - 1) / TILE_N, argmax_dev);
+  }
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) {
     c->err = std::string("tensor-core head launch: ") + cudaGetErrorString(e);
