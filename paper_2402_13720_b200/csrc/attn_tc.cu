@@ -5,32 +5,37 @@
 // described by the number of keys it sees and by where its last keys live (its own candidate's cache slots),
 // and the kernel maps "virtual positions" 0..n_vis-1 to cache slots on the fly.
 //
-// Work split.  Keys are cut by virtual position into aligned chunks of 256; one CTA handles one (kv head,
-// chunk): it stages the chunk's K and V rows in shared memory once and serves every query row and every query
-// head of the group from there, so each cached byte is read from HBM once.  Inside the CTA each of the 8 warps
-// owns 32 keys, computes S = Q K^T, a local softmax and P V with mma.sync for 16 query rows at a time, and the 8
-// warp results are folded in warp order into the chunk's (max, sum, output) triple.  A second kernel folds the
-// chunks of a row in ascending order and normalises.
+// Work split.  Keys are cut by virtual position into aligned spans of 512; one CTA handles one (kv head, span)
+// for all query rows and all query heads of the group, so every cached byte is read from HBM once.  The CTA
+// walks its span in chunks of 128 keys: K and V rows of the next chunk stream into a second shared-memory
+// buffer (cp.async) while the current one is used.  Per chunk: the 8 warps split the keys for S = Q K^T
+// (mma.sync), agree on each row's chunk maximum through shared memory, write P = exp2(S - max) as bf16 to shared
+// memory, then split the head dimension for O += P V.  Running (max, sum, O) are kept per row across the chunks
+// of the span; a second kernel folds the spans of a row in ascending order and normalises.
 //
-// Chunks below the cache length are the same for all rows.  The chunk(s) holding the block's own keys differ
-// between the trunk and each candidate: the CTA keeps the shared part of the tile and swaps in each group's own
-// rows in turn.  The value computed for a query depends only on (virtual position -> key) and on fixed chunk and
-// warp boundaries, never on the other rows of the block, so a token gets bit-identical attention whether it is
-// verified inside a candidate block or decoded alone.
+// Chunks below the cache length are the same for all rows.  A chunk holding the block's own keys differs
+// between the trunk and each candidate: it is processed once per group, with that group's keys swapped into the
+// tile and the other rows masked out (an exact no-op for them).  The value computed for a query depends only on
+// (virtual position -> key) and on fixed chunk, span and warp boundaries, never on the other rows of the block:
+// a token gets bit-identical attention whether it is verified inside a candidate block or decoded alone.
 #include "ouro_internal.h"
 
 namespace {
 
-constexpr int CH = 256;            // keys per chunk
+constexpr int CH = 128;            // keys per chunk
+constexpr int SC = 4;              // chunks per span
+constexpr int SPAN = CH * SC;
 constexpr int WARPS = 8;
-constexpr int KW = CH / WARPS;     // keys per warp
+constexpr int KW = CH / WARPS;     // keys per warp in the S phase (two 8-key MMA tiles)
 constexpr int THREADS = WARPS * 32;
+constexpr int QR = 64;             // query rows per round (4 MMA row tiles)
+constexpr int MT = QR / 16;
 
 struct AttnParams {
   const __nv_bfloat16 *q;          // [rows][H*HD] rotated queries
   const __nv_bfloat16 *k, *v;      // this layer's cache: [max_seq][Hkv*HD]
   const int32_t *lin_end, *seg_start, *seg_len, *group;
-  int rows, H, Hkv, L, cap;        // L: cache length before the block; cap: chunk slots per (row, head)
+  int rows, H, Hkv, L, cap;        // L: cache length before the block; cap: span slots per (row, head)
   float scale_log2;
   float *part;                     // [rows][H][cap][HD+2]: max (log2 domain), sum, unnormalised output
   __nv_bfloat16 *out;              // [rows][H*HD]
@@ -42,6 +47,7 @@ __device__ __forceinline__ void cp_async16(uint32_t dst, const void *src) {
 }
 __device__ __forceinline__ void cp_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
 __device__ __forceinline__ void cp_wait_all() { asm volatile("cp.async.wait_group 0;" ::: "memory"); }
+__device__ __forceinline__ void cp_wait_but_one() { asm volatile("cp.async.wait_group 1;" ::: "memory"); }
 __device__ __forceinline__ void ldsm_x4(uint32_t addr, uint32_t &r0, uint32_t &r1, uint32_t &r2, uint32_t &r3) {
   asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0, %1, %2, %3}, [%4];"
                : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(addr));
@@ -49,6 +55,9 @@ __device__ __forceinline__ void ldsm_x4(uint32_t addr, uint32_t &r0, uint32_t &r
 __device__ __forceinline__ void ldsm_x4_t(uint32_t addr, uint32_t &r0, uint32_t &r1, uint32_t &r2, uint32_t &r3) {
   asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0, %1, %2, %3}, [%4];"
                : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(addr));
+}
+__device__ __forceinline__ void ldsm_x2_t(uint32_t addr, uint32_t &r0, uint32_t &r1) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x2.trans.shared.b16 {%0, %1}, [%2];" : "=r"(r0), "=r"(r1) : "r"(addr));
 }
 __device__ __forceinline__ void mma16816(float *d, const uint32_t *a, uint32_t b0, uint32_t b1) {
   asm volatile(
@@ -60,206 +69,273 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   __nv_bfloat162 t = __floats2bfloat162_rn(lo, hi);
   return *reinterpret_cast<uint32_t *>(&t);
 }
-// log2-domain running softmax state folded with another piece: exact no-op when the piece is empty
-__device__ __forceinline__ void fold_scales(float m, float mp, float &m_new, float &a, float &b) {
-  m_new = fmaxf(m, mp);
-  a = (m == -INFINITY) ? 0.f : exp2f(m - m_new);
-  b = (mp == -INFINITY) ? 0.f : exp2f(mp - m_new);
-}
 
 template <int HD>
-__global__ void __launch_bounds__(THREADS) attn_chunk_kernel(const AttnParams p) {
-  constexpr int CPR = HD / 8;                 // 16-byte pieces per row
-  constexpr int ROWB = HD * 2;                // bytes per tile row
-  constexpr int PW = HD + 2;                  // floats per partial
+struct Smem {
+  static constexpr int ROWB = HD * 2;                              // bytes per K/V/Q tile row
+  static constexpr int KV = CH * ROWB;                             // one K or V buffer
+  static constexpr int OFF_V = 2 * KV;                             // K[2] then V[2]
+  static constexpr int OFF_Q = 4 * KV;
+  static constexpr int OFF_P = OFF_Q + QR * ROWB;                  // P: [MT][16][CH] bf16
+  static constexpr int OFF_WMAX = OFF_P + MT * 16 * CH * 2;        // [WARPS][QR]
+  static constexpr int OFF_WSUM = OFF_WMAX + WARPS * QR * 4;
+  static constexpr int OFF_NVIS = OFF_WSUM + WARPS * QR * 4;       // [OURO_MAX_ROWS]
+  static constexpr int OFF_GRP = OFF_NVIS + OURO_MAX_ROWS * 4;
+  static constexpr int BYTES = OFF_GRP + OURO_MAX_ROWS * 4;
+};
+
+template <int HD>
+__global__ void __launch_bounds__(THREADS) attn_span_kernel(const AttnParams p) {
+  using S = Smem<HD>;
+  constexpr int CPR = HD / 8;                  // 16-byte pieces per row
+  constexpr int ROWB = S::ROWB;
+  constexpr int PW = HD + 2;
+  constexpr int DW = HD / WARPS;               // output dims per warp in the P V phase (16 or 8)
+  constexpr int NT2 = DW / 8;                  // 8-dim MMA tiles per warp
   extern __shared__ __align__(128) uint8_t smem[];
-  uint8_t *Ks = smem, *Vs = smem + CH * ROWB;
-  float *mbuf = (float *)(smem + 2 * CH * ROWB);          // [WARPS][16][PW]
-  int *s_nvis = (int *)(mbuf + WARPS * 16 * PW);          // [OURO_MAX_ROWS]
+  float *wmax = (float *)(smem + S::OFF_WMAX), *wsum = (float *)(smem + S::OFF_WSUM);
+  int *s_nvis = (int *)(smem + S::OFF_NVIS), *s_grp = (int *)(smem + S::OFF_GRP);
+  const uint32_t sm_u = smem_u32(smem);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int c = blockIdx.x, kvh = blockIdx.y, c0 = c * CH;
+  const int sc = blockIdx.x, kvh = blockIdx.y;
   const int g = p.H / p.Hkv, dkv = p.Hkv * HD;
-  const uint32_t ks_u = smem_u32(Ks), vs_u = smem_u32(Vs);
-  const int key0 = warp * KW;                 // first tile row of this warp
+  const int M_all = g * p.rows;
 
-  for (int r = threadIdx.x; r < p.rows; r += THREADS) s_nvis[r] = p.lin_end[r] + p.seg_len[r];
-
-  // ---- stage the part of the chunk that every row shares (positions below the cache length); zero the rest
-  for (int idx = lane; idx < KW * CPR; idx += 32) {
-    int row = key0 + idx / CPR, ch = idx % CPR, pos = c0 + row;
-    uint32_t off = row * ROWB + ((ch ^ (row & 7)) << 4);
-    if (pos < p.L) {
-      size_t src = (size_t)pos * dkv + kvh * HD + ch * 8;
-      cp_async16(ks_u + off, p.k + src);
-      cp_async16(vs_u + off, p.v + src);
-    } else {
-      *reinterpret_cast<uint4 *>(Ks + off) = make_uint4(0, 0, 0, 0);
-      *reinterpret_cast<uint4 *>(Vs + off) = make_uint4(0, 0, 0, 0);
-    }
+  int nv_max = 0;
+  for (int r = threadIdx.x; r < p.rows; r += THREADS) {
+    s_nvis[r] = p.lin_end[r] + p.seg_len[r];
+    s_grp[r] = p.group[r];
   }
-  cp_commit();
-  __syncthreads();                            // s_nvis visible
+  __syncthreads();
+  for (int r = 0; r < p.rows; ++r) nv_max = max(nv_max, s_nvis[r]);
+  const int span0 = sc * SPAN;
+  const int n_chunks = min(SC, (nv_max - span0 + CH - 1) / CH);       // chunks of this span anybody sees
 
-  const bool common = c0 + CH <= p.L;
-  int g_begin = 0;
-  while (g_begin < p.rows) {
-    // ---- one pass: all rows (shared chunk) or the rows of one group (chunk holding block keys)
-    int g_end = p.rows, lin_g = INT_MAX, seg_g = 0;
-    if (!common) {
-      int gid = p.group[g_begin];
-      g_end = g_begin + 1;
-      while (g_end < p.rows && p.group[g_end] == gid) ++g_end;
-      int last = g_end - 1;
-      if (p.seg_len[last] > 0) { lin_g = p.lin_end[last]; seg_g = p.seg_start[last]; }
-      int nv_max = s_nvis[last];
-      if (nv_max > c0) {
-        // this group's own keys: virtual positions [max(c0, L), min(c0 + CH, nv_max)) of the warp's 32 rows
-        for (int idx = lane; idx < KW * CPR; idx += 32) {
-          int row = key0 + idx / CPR, ch = idx % CPR, pos = c0 + row;
-          if (pos >= p.L && pos < nv_max) {
-            int slot = pos < lin_g ? pos : seg_g + (pos - lin_g);
-            uint32_t off = row * ROWB + ((ch ^ (row & 7)) << 4);
-            size_t src = (size_t)slot * dkv + kvh * HD + ch * 8;
-            cp_async16(ks_u + off, p.k + src);
-            cp_async16(vs_u + off, p.v + src);
-          }
-        }
-        cp_commit();
+  // Stages the part of chunk ci every row shares (virtual positions below the cache length) and zeroes the rest.
+  auto stage_common = [&](int ci, int buf) {
+    const int c0 = span0 + ci * CH;
+    for (int idx = threadIdx.x; idx < CH * CPR; idx += THREADS) {
+      int row = idx / CPR, ch = idx % CPR, pos = c0 + row;
+      uint32_t off = buf * S::KV + row * ROWB + ((ch ^ (row & 7)) << 4);
+      if (pos < p.L) {
+        size_t src = (size_t)pos * dkv + kvh * HD + ch * 8;
+        cp_async16(sm_u + off, p.k + src);
+        cp_async16(sm_u + S::OFF_V + off, p.v + src);
+      } else {
+        *reinterpret_cast<uint4 *>(smem + off) = make_uint4(0, 0, 0, 0);
+        *reinterpret_cast<uint4 *>(smem + S::OFF_V + off) = make_uint4(0, 0, 0, 0);
       }
     }
-    cp_wait_all();
-    __syncwarp();
+    cp_commit();
+  };
 
-    const int nr = g_end - g_begin, M = g * nr;
-    for (int mt = 0; mt * 16 < M; ++mt) {
-      // the two query rows of this thread
-      const int mA = mt * 16 + (lane >> 2), mB = mA + 8;
-      const bool vA = mA < M, vB = mB < M;
-      const int rA = g_begin + (vA ? mA % nr : 0), rB = g_begin + (vB ? mB % nr : 0);
-      const int hA = kvh * g + (vA ? mA / nr : 0), hB = kvh * g + (vB ? mB / nr : 0);
-      const int nvA = vA ? s_nvis[rA] : 0, nvB = vB ? s_nvis[rB] : 0;
-      // skip tiles none of whose rows reaches this chunk (their partial is never read); same in every warp
-      if (__ballot_sync(0xffffffffu, nvA > c0 || nvB > c0) == 0) continue;
-
-      const __nv_bfloat16 *qA = p.q + (size_t)rA * p.H * HD + hA * HD + 2 * (lane & 3);
-      const __nv_bfloat16 *qB = p.q + (size_t)rB * p.H * HD + hB * HD + 2 * (lane & 3);
-      float s[4][4];
+  for (int m0 = 0; m0 < M_all; m0 += QR) {
+    // ---------------------------------------------------------------- one round of up to 64 query rows
+    // query row m -> (head m / rows, block row m % rows); rows of this thread in row tile mt: lane/4 and +8
+    int nv[2 * MT], gr[2 * MT], rr[2 * MT], hh[2 * MT];
+    bool any_row = false;
 #pragma unroll
-      for (int nt = 0; nt < 4; ++nt) s[nt][0] = s[nt][1] = s[nt][2] = s[nt][3] = 0.f;
-#pragma unroll
-      for (int ks = 0; ks < HD / 16; ++ks) {
-        uint32_t a[4];
-        a[0] = vA ? *reinterpret_cast<const uint32_t *>(qA + 16 * ks) : 0u;
-        a[1] = vB ? *reinterpret_cast<const uint32_t *>(qB + 16 * ks) : 0u;
-        a[2] = vA ? *reinterpret_cast<const uint32_t *>(qA + 16 * ks + 8) : 0u;
-        a[3] = vB ? *reinterpret_cast<const uint32_t *>(qB + 16 * ks + 8) : 0u;
-#pragma unroll
-        for (int half = 0; half < 2; ++half) {
-          int mi = lane >> 3;
-          int row = key0 + 16 * half + (lane & 7) + ((mi >> 1) << 3);
-          int ch = 2 * ks + (mi & 1);
-          uint32_t b0, b1, b2, b3;
-          ldsm_x4(ks_u + row * ROWB + ((ch ^ (row & 7)) << 4), b0, b1, b2, b3);
-          mma16816(s[2 * half], a, b0, b1);
-          mma16816(s[2 * half + 1], a, b2, b3);
-        }
-      }
-      // mask by virtual position, local softmax over this warp's 32 keys (log2 domain)
-      float mxA = -INFINITY, mxB = -INFINITY;
-#pragma unroll
-      for (int nt = 0; nt < 4; ++nt) {
-        int kp = c0 + key0 + 8 * nt + 2 * (lane & 3);
-        s[nt][0] = kp < nvA ? s[nt][0] * p.scale_log2 : -INFINITY;
-        s[nt][1] = kp + 1 < nvA ? s[nt][1] * p.scale_log2 : -INFINITY;
-        s[nt][2] = kp < nvB ? s[nt][2] * p.scale_log2 : -INFINITY;
-        s[nt][3] = kp + 1 < nvB ? s[nt][3] * p.scale_log2 : -INFINITY;
-        mxA = fmaxf(mxA, fmaxf(s[nt][0], s[nt][1]));
-        mxB = fmaxf(mxB, fmaxf(s[nt][2], s[nt][3]));
-      }
-      mxA = fmaxf(mxA, __shfl_xor_sync(0xffffffffu, mxA, 1));
-      mxA = fmaxf(mxA, __shfl_xor_sync(0xffffffffu, mxA, 2));
-      mxB = fmaxf(mxB, __shfl_xor_sync(0xffffffffu, mxB, 1));
-      mxB = fmaxf(mxB, __shfl_xor_sync(0xffffffffu, mxB, 2));
-      const float uA = mxA == -INFINITY ? 0.f : mxA, uB = mxB == -INFINITY ? 0.f : mxB;
-      float lA = 0.f, lB = 0.f;
-#pragma unroll
-      for (int nt = 0; nt < 4; ++nt) {
-        s[nt][0] = exp2f(s[nt][0] - uA);
-        s[nt][1] = exp2f(s[nt][1] - uA);
-        s[nt][2] = exp2f(s[nt][2] - uB);
-        s[nt][3] = exp2f(s[nt][3] - uB);
-        lA += s[nt][0] + s[nt][1];
-        lB += s[nt][2] + s[nt][3];
-      }
-      lA += __shfl_xor_sync(0xffffffffu, lA, 1);
-      lA += __shfl_xor_sync(0xffffffffu, lA, 2);
-      lB += __shfl_xor_sync(0xffffffffu, lB, 1);
-      lB += __shfl_xor_sync(0xffffffffu, lB, 2);
-      // O = P V over the warp's 32 keys
-      float o[HD / 8][4];
-#pragma unroll
-      for (int nt = 0; nt < HD / 8; ++nt) o[nt][0] = o[nt][1] = o[nt][2] = o[nt][3] = 0.f;
-#pragma unroll
-      for (int kk = 0; kk < 2; ++kk) {
-        uint32_t a[4];
-        a[0] = pack_bf16(s[2 * kk][0], s[2 * kk][1]);
-        a[1] = pack_bf16(s[2 * kk][2], s[2 * kk][3]);
-        a[2] = pack_bf16(s[2 * kk + 1][0], s[2 * kk + 1][1]);
-        a[3] = pack_bf16(s[2 * kk + 1][2], s[2 * kk + 1][3]);
-#pragma unroll
-        for (int np = 0; np < HD / 16; ++np) {
-          int mi = lane >> 3;
-          int row = key0 + 16 * kk + (lane & 7) + ((mi & 1) << 3);
-          int ch = 2 * np + (mi >> 1);
-          uint32_t b0, b1, b2, b3;
-          ldsm_x4_t(vs_u + row * ROWB + ((ch ^ (row & 7)) << 4), b0, b1, b2, b3);
-          mma16816(o[2 * np], a, b0, b1);
-          mma16816(o[2 * np + 1], a, b2, b3);
-        }
-      }
-      // park the warp's piece, then fold the 8 pieces in warp order
-      float *mineA = mbuf + ((size_t)warp * 16 + (lane >> 2)) * PW, *mineB = mineA + 8 * PW;
-      if ((lane & 3) == 0) { mineA[0] = mxA; mineA[1] = lA; mineB[0] = mxB; mineB[1] = lB; }
-#pragma unroll
-      for (int nt = 0; nt < HD / 8; ++nt) {
-        int d = 2 + 8 * nt + 2 * (lane & 3);
-        mineA[d] = o[nt][0]; mineA[d + 1] = o[nt][1];
-        mineB[d] = o[nt][2]; mineB[d + 1] = o[nt][3];
-      }
-      __syncthreads();
-      {
-        constexpr int DPT = HD / 16;                 // output dims per thread
-        const int row = threadIdx.x >> 4, d0 = (threadIdx.x & 15) * DPT;
-        const int m = mt * 16 + row;
-        if (m < M) {
-          float mr = -INFINITY, lr = 0.f, acc[DPT];
-#pragma unroll
-          for (int i = 0; i < DPT; ++i) acc[i] = 0.f;
-#pragma unroll
-          for (int w = 0; w < WARPS; ++w) {
-            const float *pc = mbuf + ((size_t)w * 16 + row) * PW;
-            float mn, a, b;
-            fold_scales(mr, pc[0], mn, a, b);
-            lr = lr * a + pc[1] * b;
-#pragma unroll
-            for (int i = 0; i < DPT; ++i) acc[i] = acc[i] * a + pc[2 + d0 + i] * b;
-            mr = mn;
-          }
-          const int r = g_begin + m % nr, head = kvh * g + m / nr;
-          float *dst = p.part + (((size_t)r * p.H + head) * p.cap + c) * PW;
-          if ((threadIdx.x & 15) == 0) { dst[0] = mr; dst[1] = lr; }
-#pragma unroll
-          for (int i = 0; i < DPT; ++i) dst[2 + d0 + i] = acc[i];
-        }
-      }
-      __syncthreads();
+    for (int i = 0; i < 2 * MT; ++i) {
+      int m = m0 + (i >> 1) * 16 + (lane >> 2) + (i & 1) * 8;
+      bool ok = m < M_all;
+      rr[i] = ok ? m % p.rows : 0;
+      hh[i] = kvh * g + (ok ? m / p.rows : 0);
+      nv[i] = ok ? s_nvis[rr[i]] : 0;
+      gr[i] = ok ? s_grp[rr[i]] : -1;
+      any_row = any_row || nv[i] > span0;
     }
-    g_begin = g_end;
+    if (!__syncthreads_or(any_row)) continue;          // nobody in this round reaches the span
+
+    __syncthreads();                                    // previous round done with every buffer
+    for (int idx = threadIdx.x; idx < QR * CPR; idx += THREADS) {
+      int row = idx / CPR, ch = idx % CPR, m = m0 + row;
+      uint32_t off = S::OFF_Q + row * ROWB + ((ch ^ (row & 7)) << 4);
+      if (m < M_all)
+        cp_async16(sm_u + off, p.q + (size_t)(m % p.rows) * p.H * HD + (kvh * g + m / p.rows) * HD + ch * 8);
+      else
+        *reinterpret_cast<uint4 *>(smem + off) = make_uint4(0, 0, 0, 0);
+    }
+    stage_common(0, 0);                                 // one group: Q and chunk 0
+
+    float o[MT][NT2][4], m_run[2 * MT], l_run[2 * MT];
+#pragma unroll
+    for (int i = 0; i < 2 * MT; ++i) { m_run[i] = -INFINITY; l_run[i] = 0.f; }
+#pragma unroll
+    for (int mt = 0; mt < MT; ++mt)
+#pragma unroll
+      for (int nt = 0; nt < NT2; ++nt) o[mt][nt][0] = o[mt][nt][1] = o[mt][nt][2] = o[mt][nt][3] = 0.f;
+
+    for (int ci = 0; ci < n_chunks; ++ci) {
+      const int buf = ci & 1, c0 = span0 + ci * CH;
+      if (ci + 1 < n_chunks) { stage_common(ci + 1, buf ^ 1); cp_wait_but_one(); } else { cp_wait_all(); }
+      __syncthreads();
+      const bool common = c0 + CH <= p.L;
+      int g_begin = 0;
+      while (g_begin < p.rows) {
+        // -------------------------------------------------------------- one pass over the chunk
+        int g_end = p.rows, gid = -2;                  // gid -2: every row takes part
+        if (!common) {
+          gid = s_grp[g_begin];
+          g_end = g_begin + 1;
+          while (g_end < p.rows && s_grp[g_end] == gid) ++g_end;
+          const int last = g_end - 1, nvg = s_nvis[last];
+          int lin_g = INT_MAX, seg_g = 0;
+          if (p.seg_len[last] > 0) { lin_g = p.lin_end[last]; seg_g = p.seg_start[last]; }
+          bool mine = false;
+#pragma unroll
+          for (int i = 0; i < 2 * MT; ++i) mine = mine || (gr[i] == gid && nv[i] > c0);
+          if (!__syncthreads_or(mine)) { g_begin = g_end; continue; }   // no row of this round in the group
+          // swap in the group's own keys: virtual positions [max(c0, L), min(c0 + CH, nvg))
+          for (int idx = threadIdx.x; idx < CH * CPR; idx += THREADS) {
+            int row = idx / CPR, ch = idx % CPR, pos = c0 + row;
+            if (pos >= p.L && pos < nvg) {
+              int slot = pos < lin_g ? pos : seg_g + (pos - lin_g);
+              uint32_t off = buf * S::KV + row * ROWB + ((ch ^ (row & 7)) << 4);
+              size_t src = (size_t)slot * dkv + kvh * HD + ch * 8;
+              cp_async16(sm_u + off, p.k + src);
+              cp_async16(sm_u + S::OFF_V + off, p.v + src);
+            }
+          }
+          cp_commit();
+          cp_wait_all();
+          __syncthreads();
+        }
+        // ---- S = Q K^T for this warp's 16 keys, all row tiles
+        float s[MT][2][4];
+#pragma unroll
+        for (int mt = 0; mt < MT; ++mt)
+#pragma unroll
+          for (int nt = 0; nt < 2; ++nt) s[mt][nt][0] = s[mt][nt][1] = s[mt][nt][2] = s[mt][nt][3] = 0.f;
+        const uint32_t k_u = sm_u + buf * S::KV, v_u = sm_u + S::OFF_V + buf * S::KV;
+#pragma unroll
+        for (int ks = 0; ks < HD / 16; ++ks) {
+          const int mi = lane >> 3;
+          uint32_t b0, b1, b2, b3;
+          {
+            int row = warp * KW + (lane & 7) + ((mi >> 1) << 3), ch = 2 * ks + (mi & 1);
+            ldsm_x4(k_u + row * ROWB + ((ch ^ (row & 7)) << 4), b0, b1, b2, b3);
+          }
+#pragma unroll
+          for (int mt = 0; mt < MT; ++mt) {
+            uint32_t a[4];
+            int row = mt * 16 + (lane & 7) + ((mi & 1) << 3), ch = 2 * ks + (mi >> 1);
+            ldsm_x4(sm_u + S::OFF_Q + row * ROWB + ((ch ^ (row & 7)) << 4), a[0], a[1], a[2], a[3]);
+            mma16816(s[mt][0], a, b0, b1);
+            mma16816(s[mt][1], a, b2, b3);
+          }
+        }
+        // ---- mask by virtual position and group; warp-local row maxima (log2 domain)
+#pragma unroll
+        for (int mt = 0; mt < MT; ++mt) {
+          const int iA = 2 * mt, iB = 2 * mt + 1;
+          const int nA = (gid == -2 || gr[iA] == gid) ? nv[iA] : 0, nB = (gid == -2 || gr[iB] == gid) ? nv[iB] : 0;
+          float mxA = -INFINITY, mxB = -INFINITY;
+#pragma unroll
+          for (int nt = 0; nt < 2; ++nt) {
+            int kp = c0 + warp * KW + 8 * nt + 2 * (lane & 3);
+            s[mt][nt][0] = kp < nA ? s[mt][nt][0] * p.scale_log2 : -INFINITY;
+            s[mt][nt][1] = kp + 1 < nA ? s[mt][nt][1] * p.scale_log2 : -INFINITY;
+            s[mt][nt][2] = kp < nB ? s[mt][nt][2] * p.scale_log2 : -INFINITY;
+            s[mt][nt][3] = kp + 1 < nB ? s[mt][nt][3] * p.scale_log2 : -INFINITY;
+            mxA = fmaxf(mxA, fmaxf(s[mt][nt][0], s[mt][nt][1]));
+            mxB = fmaxf(mxB, fmaxf(s[mt][nt][2], s[mt][nt][3]));
+          }
+          mxA = fmaxf(mxA, __shfl_xor_sync(0xffffffffu, mxA, 1));
+          mxA = fmaxf(mxA, __shfl_xor_sync(0xffffffffu, mxA, 2));
+          mxB = fmaxf(mxB, __shfl_xor_sync(0xffffffffu, mxB, 1));
+          mxB = fmaxf(mxB, __shfl_xor_sync(0xffffffffu, mxB, 2));
+          if ((lane & 3) == 0) {
+            wmax[warp * QR + mt * 16 + (lane >> 2)] = mxA;
+            wmax[warp * QR + mt * 16 + (lane >> 2) + 8] = mxB;
+          }
+        }
+        __syncthreads();
+        // ---- new running maximum, P = exp2(S - max) to shared memory, warp-local row sums
+        float scale_old[2 * MT];
+#pragma unroll
+        for (int mt = 0; mt < MT; ++mt) {
+#pragma unroll
+          for (int hb = 0; hb < 2; ++hb) {
+            const int i = 2 * mt + hb, row = mt * 16 + (lane >> 2) + 8 * hb;
+            float mc = wmax[row];
+#pragma unroll
+            for (int w = 1; w < WARPS; ++w) mc = fmaxf(mc, wmax[w * QR + row]);
+            const float mn = fmaxf(m_run[i], mc);
+            scale_old[i] = (m_run[i] == -INFINITY) ? 0.f : exp2f(m_run[i] - mn);   // mn finite whenever m_run is
+            m_run[i] = mn;
+            const float use = mn == -INFINITY ? 0.f : mn;
+            float sum = 0.f;
+#pragma unroll
+            for (int nt = 0; nt < 2; ++nt) {
+              float p0 = exp2f(s[mt][nt][2 * hb] - use), p1 = exp2f(s[mt][nt][2 * hb + 1] - use);
+              sum += p0 + p1;
+              int ch = warp * 2 + nt;                               // 16-byte piece: keys 8*ch .. 8*ch+7
+              uint32_t off = S::OFF_P + (mt * 16 + (row & 15)) * (CH * 2) + ((ch ^ (row & 7)) << 4) + 4 * (lane & 3);
+              *reinterpret_cast<uint32_t *>(smem + off) = pack_bf16(p0, p1);
+            }
+            sum += __shfl_xor_sync(0xffffffffu, sum, 1);
+            sum += __shfl_xor_sync(0xffffffffu, sum, 2);
+            if ((lane & 3) == 0) wsum[warp * QR + row] = sum;
+          }
+        }
+        __syncthreads();
+        // ---- running sums and O = O * scale + P V for this warp's slice of the head dimension
+#pragma unroll
+        for (int i = 0; i < 2 * MT; ++i) {
+          const int row = (i >> 1) * 16 + (lane >> 2) + 8 * (i & 1);
+          float add = wsum[row];
+#pragma unroll
+          for (int w = 1; w < WARPS; ++w) add += wsum[w * QR + row];
+          l_run[i] = l_run[i] * scale_old[i] + add;
+        }
+#pragma unroll
+        for (int mt = 0; mt < MT; ++mt)
+#pragma unroll
+          for (int nt = 0; nt < NT2; ++nt) {
+            o[mt][nt][0] *= scale_old[2 * mt]; o[mt][nt][1] *= scale_old[2 * mt];
+            o[mt][nt][2] *= scale_old[2 * mt + 1]; o[mt][nt][3] *= scale_old[2 * mt + 1];
+          }
+#pragma unroll
+        for (int kk = 0; kk < CH / 16; ++kk) {
+          const int mi = lane >> 3;
+          uint32_t b0, b1, b2 = 0, b3 = 0;
+          if (NT2 == 2) {
+            int row = 16 * kk + (lane & 7) + ((mi & 1) << 3), ch = warp * 2 + (mi >> 1);
+            ldsm_x4_t(v_u + row * ROWB + ((ch ^ (row & 7)) << 4), b0, b1, b2, b3);
+          } else {
+            int row = 16 * kk + (lane & 7) + ((mi & 1) << 3), ch = warp;
+            ldsm_x2_t(v_u + row * ROWB + ((ch ^ (row & 7)) << 4), b0, b1);
+          }
+#pragma unroll
+          for (int mt = 0; mt < MT; ++mt) {
+            uint32_t a[4];
+            int row = (lane & 7) + ((mi & 1) << 3), ch = 2 * kk + (mi >> 1);
+            ldsm_x4(sm_u + S::OFF_P + (mt * 16 + row) * (CH * 2) + ((ch ^ (row & 7)) << 4), a[0], a[1], a[2], a[3]);
+            mma16816(o[mt][0], a, b0, b1);
+            if (NT2 == 2) mma16816(o[mt][NT2 - 1], a, b2, b3);
+          }
+        }
+        __syncthreads();                              // wmax, wsum, P and the tile may change now
+        g_begin = g_end;
+      }
+    }
+    // ---- the span's piece of every row of the round that reaches it
+#pragma unroll
+    for (int i = 0; i < 2 * MT; ++i) {
+      if (nv[i] <= span0) continue;
+      float *dst = p.part + (((size_t)rr[i] * p.H + hh[i]) * p.cap + sc) * PW;
+      if (warp == 0 && (lane & 3) == 0) { dst[0] = m_run[i]; dst[1] = l_run[i]; }
+#pragma unroll
+      for (int nt = 0; nt < NT2; ++nt) {
+        int d = warp * DW + 8 * nt + 2 * (lane & 3);
+        *reinterpret_cast<float2 *>(dst + 2 + d) = make_float2(o[i >> 1][nt][2 * (i & 1)], o[i >> 1][nt][2 * (i & 1) + 1]);
+      }
+    }
   }
 }
 
-// Folds a row's chunks in ascending order and normalises.  One warp per (row, head).
+// Folds a row's spans in ascending order and normalises.  One warp per (row, head).
 template <int HD>
 __global__ void attn_merge_kernel(const AttnParams p) {
   constexpr int PW = HD + 2, DPL = HD / 32;
@@ -267,15 +343,15 @@ __global__ void attn_merge_kernel(const AttnParams p) {
   const int r = blockIdx.x, head = blockIdx.y * (blockDim.x >> 5) + warp;
   if (head >= p.H) return;
   const int nv = p.lin_end[r] + p.seg_len[r];
-  const int nc = (nv + CH - 1) / CH;
+  const int ns = (nv + SPAN - 1) / SPAN;
   const float *src = p.part + ((size_t)r * p.H + head) * p.cap * PW;
   float m = -INFINITY, l = 0.f, acc[DPL];
 #pragma unroll
   for (int i = 0; i < DPL; ++i) acc[i] = 0.f;
-  for (int c = 0; c < nc; ++c) {
+  for (int c = 0; c < ns; ++c) {
     const float *pc = src + (size_t)c * PW;
-    float mn, a, b;
-    fold_scales(m, pc[0], mn, a, b);
+    const float mp = pc[0], mn = fmaxf(m, mp);
+    const float a = (m == -INFINITY) ? 0.f : exp2f(m - mn), b = (mp == -INFINITY) ? 0.f : exp2f(mp - mn);
     l = l * a + pc[1] * b;
 #pragma unroll
     for (int i = 0; i < DPL; ++i) acc[i] = acc[i] * a + pc[2 + lane + 32 * i] * b;
@@ -286,28 +362,25 @@ __global__ void attn_merge_kernel(const AttnParams p) {
   for (int i = 0; i < DPL; ++i) p.out[(size_t)r * p.H * HD + head * HD + lane + 32 * i] = __float2bfloat16_rn(acc[i] * inv);
 }
 
-template <int HD>
-size_t chunk_smem() { return (size_t)2 * CH * HD * 2 + (size_t)WARPS * 16 * (HD + 2) * 4 + OURO_MAX_ROWS * 4; }
-
 }  // namespace
 
 bool attention_tc_supported(const ouro_model_desc &d) { return d.dtype == OURO_BF16 && (d.head_dim == 64 || d.head_dim == 128); }
 
 size_t attention_tc_scratch_bytes(const ouro_model_desc &d) {
   if (!attention_tc_supported(d)) return 0;
-  size_t cap = (d.max_seq + CH - 1) / CH;
+  size_t cap = (d.max_seq + SPAN - 1) / SPAN;
   return (size_t)OURO_MAX_ROWS * d.n_heads * cap * (d.head_dim + 2) * sizeof(float);
 }
 
 int attention_tc_setup() {
-  if (cudaFuncSetAttribute(attn_chunk_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)chunk_smem<128>()) != cudaSuccess)
+  if (cudaFuncSetAttribute(attn_span_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, Smem<128>::BYTES) != cudaSuccess)
     return OURO_ECUDA;
-  if (cudaFuncSetAttribute(attn_chunk_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)chunk_smem<64>()) != cudaSuccess)
+  if (cudaFuncSetAttribute(attn_span_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, Smem<64>::BYTES) != cudaSuccess)
     return OURO_ECUDA;
   return OURO_OK;
 }
 
-// n_vis_max: the largest number of visible keys over the block's rows (cache length + rows at most).
+// n_vis_max: an upper bound of the number of keys any row of the block sees (cache length + rows).
 void launch_attention_tc(const ouro_model_desc &d, const void *q, const void *k_cache, const void *v_cache, const BlockDev &b,
                          int rows, int L, int n_vis_max, int layer, float *part, void *out, cudaStream_t s) {
   OURO_COUNT_LAUNCH();
@@ -319,16 +392,16 @@ void launch_attention_tc(const ouro_model_desc &d, const void *q, const void *k_
   p.v = (const __nv_bfloat16 *)v_cache + off;
   p.lin_end = b.lin_end; p.seg_start = b.seg_start; p.seg_len = b.seg_len; p.group = b.group;
   p.rows = rows; p.H = d.n_heads; p.Hkv = d.n_kv_heads; p.L = L;
-  p.cap = (d.max_seq + CH - 1) / CH;
+  p.cap = (d.max_seq + SPAN - 1) / SPAN;
   p.scale_log2 = 1.4426950408889634f / sqrtf((float)d.head_dim);
   p.part = part;
   p.out = (__nv_bfloat16 *)out;
-  dim3 grid((n_vis_max + CH - 1) / CH, d.n_kv_heads), mgrid(rows, (d.n_heads + 3) / 4);
+  dim3 grid((n_vis_max + SPAN - 1) / SPAN, d.n_kv_heads), mgrid(rows, (d.n_heads + 3) / 4);
   if (d.head_dim == 128) {
-    attn_chunk_kernel<128><<<grid, THREADS, chunk_smem<128>(), s>>>(p);
+    attn_span_kernel<128><<<grid, THREADS, Smem<128>::BYTES, s>>>(p);
     attn_merge_kernel<128><<<mgrid, 128, 0, s>>>(p);
   } else {
-    attn_chunk_kernel<64><<<grid, THREADS, chunk_smem<64>(), s>>>(p);
+    attn_span_kernel<64><<<grid, THREADS, Smem<64>::BYTES, s>>>(p);
     attn_merge_kernel<64><<<mgrid, 128, 0, s>>>(p);
   }
 }
