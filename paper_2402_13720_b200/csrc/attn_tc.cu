@@ -97,6 +97,8 @@ __global__ void __launch_bounds__(THREADS) attn_span_kernel(const AttnParams p) 
   int *s_nvis = (int *)(smem + S::OFF_NVIS), *s_grp = (int *)(smem + S::OFF_GRP);
   const uint32_t sm_u = smem_u32(smem);
 
+  pdl_trigger();
+  pdl_wait();
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int sc = blockIdx.x, kvh = blockIdx.y;
   const int g = p.H / p.Hkv, dkv = p.Hkv * HD;
@@ -339,6 +341,8 @@ __global__ void __launch_bounds__(THREADS) attn_span_kernel(const AttnParams p) 
 template <int HD>
 __global__ void attn_merge_kernel(const AttnParams p) {
   constexpr int PW = HD + 2, DPL = HD / 32;
+  pdl_trigger();
+  pdl_wait();
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int r = blockIdx.x, head = blockIdx.y * (blockDim.x >> 5) + warp;
   if (head >= p.H) return;
@@ -398,10 +402,10 @@ void launch_attention_tc(const ouro_model_desc &d, const void *q, const void *k_
   p.out = (__nv_bfloat16 *)out;
   dim3 grid((n_vis_max + SPAN - 1) / SPAN, d.n_kv_heads), mgrid(rows, (d.n_heads + 3) / 4);
   if (d.head_dim == 128) {
-    attn_span_kernel<128><<<grid, THREADS, Smem<128>::BYTES, s>>>(p);
-    attn_merge_kernel<128><<<mgrid, 128, 0, s>>>(p);
+    launch_pdl(attn_span_kernel<128>, grid, THREADS, Smem<128>::BYTES, s, p);
+    launch_pdl(attn_merge_kernel<128>, mgrid, 128, 0, s, p);
   } else {
-    attn_span_kernel<64><<<grid, THREADS, Smem<64>::BYTES, s>>>(p);
-    attn_merge_kernel<64><<<mgrid, 128, 0, s>>>(p);
+    launch_pdl(attn_span_kernel<64>, grid, THREADS, Smem<64>::BYTES, s, p);
+    launch_pdl(attn_merge_kernel<64>, mgrid, 128, 0, s, p);
   }
 }

@@ -26,7 +26,7 @@ namespace {
 constexpr int TILE_N = 128;       // weight rows per tile (MMA M)
 constexpr int BLOCK_K = 64;       // bf16 elements per k-block: one 128-byte swizzle row
 constexpr int A_BYTES = TILE_N * BLOCK_K * 2;
-constexpr int THREADS = 192;      // warp 0 TMA, warp 1 MMA, warps 2..5 epilogue
+constexpr int THREADS = 224;      // warp 0 weight TMA, warp 1 MMA, warps 2..5 epilogue, warp 6 activation TMA
 constexpr int MAX_GRID = 160;
 constexpr int SLOT_FLOATS = TILE_N * OURO_MAX_ROWS;
 constexpr uint32_t SPIN_LIMIT = 1u << 24;
@@ -37,7 +37,7 @@ enum { MODE_STORE = 0, MODE_RESIDUAL = 1, MODE_SWIGLU = 2, MODE_HEAD = 3 };   //
 
 struct GemmParams {
   CUtensorMap a[3];   // weight matrices stacked along the output dimension (q|k|v), or gate and up
-  CUtensorMap b;      // activations, box = 64 x 16
+  CUtensorMap b;      // activations, box = 64 x t_pad
   int a_tiles[3];     // tiles of each stacked matrix (MODE_STORE / MODE_RESIDUAL)
   int a_rows[3];      // output features of each stacked matrix
   int a_count;
@@ -210,12 +210,13 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_tc_kernel(const __grid_consta
   int *last_flag = (int *)(bars + 38);
   volatile int *wait_flag = (volatile int *)(bars + 39);   // [2]: outcome of the epilogue's accumulator wait
 
+  pdl_trigger();
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int acc_cols = p.t_pad <= 32 ? 32 : p.t_pad <= 64 ? 64 : 128;   // columns per accumulator buffer
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < p.stages; ++s) {
-      mbar_init(&full[s], 1);
+      mbar_init(&full[s], 2);          // weight producer + activation producer, each with its byte count
       mbar_init(&empty[s], 1);
     }
     for (int a = 0; a < 2; ++a) {
@@ -238,27 +239,49 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_tc_kernel(const __grid_consta
   if (warp == 0) {
     // ---------------------------------------------------------------- TMA producer
     if (lane == 0) {
+      // The weights do not depend on the previous kernel, so this warp never waits for it: the ring fills with
+      // weight tiles while the predecessor drains.  The activation tiles come from warp 6, after its wait.
+      auto issue = [&](const Span &s, int kb, int st) {
+        uint8_t *sa = ring + (size_t)st * stage_bytes;
+        mbar_expect_tx(&full[st], A_BYTES);
+        if (p.mode == MODE_SWIGLU) {
+          tma_load_2d(sa, &p.a[0], &full[st], kb * BLOCK_K, s.tile * 64, HINT_EVICT_FIRST);
+          tma_load_2d(sa + A_BYTES / 2, &p.a[1], &full[st], kb * BLOCK_K, s.tile * 64, HINT_EVICT_FIRST);
+        } else {
+          int seg, row0, col0, valid;
+          locate(p, s.tile, seg, row0, col0, valid);
+          tma_load_2d(sa, &p.a[seg], &full[st], kb * BLOCK_K, row0, HINT_EVICT_FIRST);
+        }
+      };
       SpanWalker w(p);
       Span s;
       uint32_t n = 0;
       bool ok = true;
       while (ok && w.next(s)) {
-        int seg, row0, col0, valid;
-        if (p.mode == MODE_SWIGLU) { seg = 0; row0 = s.tile * 64; } else locate(p, s.tile, seg, row0, col0, valid);
         for (int kb = s.kb0; kb < s.kb1 && ok; ++kb, ++n) {
           int st = n % p.stages;
           if (n >= (uint32_t)p.stages) ok = mbar_wait(&empty[st], ((n / p.stages) - 1) & 1) && !*abort_flag;
           if (!ok) break;
-          uint8_t *sa = ring + (size_t)st * stage_bytes, *sb = sa + A_BYTES;
-          mbar_expect_tx(&full[st], stage_bytes);
-          if (p.mode == MODE_SWIGLU) {
-            tma_load_2d(sa, &p.a[0], &full[st], kb * BLOCK_K, row0, HINT_EVICT_FIRST);
-            tma_load_2d(sa + A_BYTES / 2, &p.a[1], &full[st], kb * BLOCK_K, row0, HINT_EVICT_FIRST);
-          } else {
-            tma_load_2d(sa, &p.a[seg], &full[st], kb * BLOCK_K, row0, HINT_EVICT_FIRST);
-          }
-          for (int r = 0; r < p.t_pad; r += 16)
-            tma_load_2d(sb + r * BLOCK_K * 2, &p.b, &full[st], kb * BLOCK_K, r, HINT_EVICT_LAST);
+          issue(s, kb, st);
+        }
+      }
+      if (!ok) { *abort_flag = 1; atomicExch(p.status, 1); }
+    }
+  } else if (warp == 6) {
+    // ---------------------------------------------------------------- activation producer
+    if (lane == 0) {
+      pdl_wait();                                  // the activations are the previous kernel's output
+      SpanWalker w(p);
+      Span s;
+      uint32_t n = 0;
+      bool ok = true;
+      while (ok && w.next(s)) {
+        for (int kb = s.kb0; kb < s.kb1 && ok; ++kb, ++n) {
+          int st = n % p.stages;
+          if (n >= (uint32_t)p.stages) ok = mbar_wait(&empty[st], ((n / p.stages) - 1) & 1) && !*abort_flag;
+          if (!ok) break;
+          mbar_expect_tx(&full[st], b_bytes);
+          tma_load_2d(ring + (size_t)st * stage_bytes + A_BYTES, &p.b, &full[st], kb * BLOCK_K, 0, HINT_EVICT_LAST);
         }
       }
       if (!ok) { *abort_flag = 1; atomicExch(p.status, 1); }
@@ -296,6 +319,7 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_tc_kernel(const __grid_consta
     }
   } else {
     // ---------------------------------------------------------------- epilogue warps
+    pdl_wait();
     const int q = warp & 3;                      // TMEM lane quarter this warp may read
     const int nl = q * 32 + lane;                // row of the tile held by this thread
     const int et = threadIdx.x - 64;             // 0..127 among the epilogue threads
@@ -547,7 +571,8 @@ struct LayerMaps {
 struct FastModel {
   bool ok = false;
   std::vector<LayerMaps> layers;
-  CUtensorMap head, x_d, x_q, x_f;   // activations: normed [128, d], attention out [128, dq], SwiGLU out [128, F]
+  CUtensorMap head;
+  CUtensorMap x_d[8], x_q[8], x_f[8];   // activations normed [128, d], attention out [128, dq], SwiGLU out [128, F]; box rows 16, 32, .., 128
 };
 struct FastState {
   FastModel m[2];
@@ -637,9 +662,11 @@ int ouro_fast_setup(ouro_ctx *c) {
            make_map(&lm.wg, M.w_gate[l], d.d_ffn, d.d_model, 64) && make_map(&lm.wu, M.w_up[l], d.d_ffn, d.d_model, 64) &&
            make_map(&lm.wd, M.w_down[l], d.d_model, d.d_ffn, TILE_N);
     }
-    ok = ok && make_map(&fm.head, M.lm_head, d.vocab, d.d_model, TILE_N) &&
-         make_map(&fm.x_d, c->a.xn, OURO_MAX_ROWS, d.d_model, 16) && make_map(&fm.x_q, c->a.att, OURO_MAX_ROWS, dq, 16) &&
-         make_map(&fm.x_f, c->a.act, OURO_MAX_ROWS, d.d_ffn, 16);
+    ok = ok && make_map(&fm.head, M.lm_head, d.vocab, d.d_model, TILE_N);
+    for (int i = 0; i < 8 && ok; ++i)
+      ok = make_map(&fm.x_d[i], c->a.xn, OURO_MAX_ROWS, d.d_model, 16 * (i + 1)) &&
+           make_map(&fm.x_q[i], c->a.att, OURO_MAX_ROWS, dq, 16 * (i + 1)) &&
+           make_map(&fm.x_f[i], c->a.act, OURO_MAX_ROWS, d.d_ffn, 16 * (i + 1));
     if (!ok) {
       delete f;
       c->err = "cuTensorMapEncodeTiled failed";
@@ -656,19 +683,20 @@ void ouro_fast_teardown(ouro_ctx *c) {
   c->fast = nullptr;
 }
 
-static void launch_gemm_tc(ouro_ctx *c, GemmParams &p, int K, int rows) {
+static void launch_gemm_tc(ouro_ctx *c, GemmParams &p, const CUtensorMap *xmaps, int K, int rows) {
   OURO_COUNT_LAUNCH();
   FastState &s = c->fast->s;
   p.kb = K / BLOCK_K;
   p.rows = rows;
   p.t_pad = (rows + 15) & ~15;
+  p.b = xmaps[p.t_pad / 16 - 1];
   p.stages = stages_for(p.t_pad, s.smem_max);
   p.scratch = s.slots;
   p.counters = s.counters;
   p.status = &c->st->status;
   int total = p.tiles * p.kb;
   int grid = total < s.grid ? total : s.grid;
-  gemm_tc_kernel<<<grid, THREADS, s.smem_max, c->stream>>>(p);
+  launch_pdl(gemm_tc_kernel, grid, THREADS, (size_t)s.smem_max, c->stream, p);
 }
 
 // One decoder layer with the tensor-core GEMMs; OURO_ESTATE when the model does not qualify.
@@ -690,12 +718,11 @@ int ouro_fast_layer(ouro_ctx *c, int which, int l, int rows) {
     p.a_tiles[0] = tiles(dq); p.a_tiles[1] = tiles(dkv); p.a_tiles[2] = tiles(dkv);
     p.a_rows[0] = dq; p.a_rows[1] = dkv; p.a_rows[2] = dkv;
     p.a_count = 3;
-    p.b = fm.x_d;
     p.mode = MODE_STORE;
     p.tiles = p.a_tiles[0] + p.a_tiles[1] + p.a_tiles[2];
     p.out_f32 = a.qkv;
     p.ldo = dq + 2 * dkv;
-    launch_gemm_tc(c, p, d.d_model, rows);
+    launch_gemm_tc(c, p, fm.x_d, d.d_model, rows);
   }
   { ProfScope ps(c, OURO_PROF_ROPE); launch_rope_append(d, a.qkv, M.blk.pos, M.rope_cos, M.rope_sin, rows, M.L, l, a.q, M.k_cache, M.v_cache, s); }
   {
@@ -709,34 +736,31 @@ int ouro_fast_layer(ouro_ctx *c, int which, int l, int rows) {
     ProfScope ps(c, OURO_PROF_WO);
     GemmParams p{};
     p.a[0] = lm.wo; p.a_tiles[0] = tiles(d.d_model); p.a_rows[0] = d.d_model; p.a_count = 1;
-    p.b = fm.x_q;
     p.mode = MODE_RESIDUAL;
     p.tiles = p.a_tiles[0];
     p.out_f32 = a.x;
     p.ldo = d.d_model;
-    launch_gemm_tc(c, p, dq, rows);
+    launch_gemm_tc(c, p, fm.x_q, dq, rows);
   }
   { ProfScope ps(c, OURO_PROF_NORM); launch_rmsnorm(OURO_BF16, a.x, M.ffn_norm[l], rows, d.d_model, d.rms_eps, a.xn, s); }
   {
     ProfScope ps(c, OURO_PROF_GATEUP);
     GemmParams p{};
     p.a[0] = lm.wg; p.a[1] = lm.wu; p.a_rows[0] = d.d_ffn; p.a_count = 2;
-    p.b = fm.x_d;
     p.mode = MODE_SWIGLU;
     p.tiles = (d.d_ffn + 63) / 64;
     p.out_bf16 = (__nv_bfloat16 *)a.act;
-    launch_gemm_tc(c, p, d.d_model, rows);
+    launch_gemm_tc(c, p, fm.x_d, d.d_model, rows);
   }
   {
     ProfScope ps(c, OURO_PROF_DOWN);
     GemmParams p{};
     p.a[0] = lm.wd; p.a_tiles[0] = tiles(d.d_model); p.a_rows[0] = d.d_model; p.a_count = 1;
-    p.b = fm.x_f;
     p.mode = MODE_RESIDUAL;
     p.tiles = p.a_tiles[0];
     p.out_f32 = a.x;
     p.ldo = d.d_model;
-    launch_gemm_tc(c, p, d.d_ffn, rows);
+    launch_gemm_tc(c, p, fm.x_f, d.d_ffn, rows);
   }
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) {
@@ -749,6 +773,8 @@ int ouro_fast_layer(ouro_ctx *c, int which, int l, int rows) {
 // Final norm, LM head and greedy choice.  The GEMM's epilogue keeps, per 128-entry vocabulary tile, each
 // token's best logit and index; a small kernel then picks the best tile per token.  logits may be NULL.
 __global__ void argmax_tiles_kernel(const float *tile_max, const int *tile_arg, int tiles, int32_t *out) {
+  pdl_trigger();
+  pdl_wait();
   const int t = blockIdx.x;
   float bv = -INFINITY;
   int bi = INT_MAX;
@@ -784,19 +810,19 @@ int ouro_fast_head(ouro_ctx *c, int which, int rows, float *logits, int32_t *arg
     ProfScope ps(c, OURO_PROF_HEAD);
     GemmParams p{};
     p.a[0] = fm.head; p.a_tiles[0] = (d.vocab + TILE_N - 1) / TILE_N; p.a_rows[0] = d.vocab; p.a_count = 1;
-    p.b = fm.x_d;
     p.mode = MODE_HEAD;
     p.tiles = p.a_tiles[0];
     p.out_f32 = logits;
     p.ldo = d.vocab;
     p.tile_max = c->fast->s.tile_max;
     p.tile_arg = c->fast->s.tile_arg;
-    launch_gemm_tc(c, p, d.d_model, rows);
+    launch_gemm_tc(c, p, fm.x_d, d.d_model, rows);
   }
   {
     ProfScope ps(c, OURO_PROF_ARGMAX);
     OURO_COUNT_LAUNCH();
-    argmax_tiles_kernel<<<rows, 128, 0, c->stream>>>(c->fast->s.tile_max, c->fast->s.tile_arg, (d.vocab + TILE_N - 1) / TILE_N, argmax_dev);
+    launch_pdl(argmax_tiles_kernel, rows, 128, 0, c->stream, (const float *)c->fast->s.tile_max, (const int *)c->fast->s.tile_arg,
+               (int)((d.vocab + TILE_N - 1) / TILE_N), argmax_dev);
   }
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) {

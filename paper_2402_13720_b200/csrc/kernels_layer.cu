@@ -65,20 +65,24 @@ void launch_rope_table(float *cos_t, float *sin_t, int max_seq, int head_dim, fl
 // --------------------------------------------------------------------------------- embedding
 template <typename T>
 __global__ void embed_kernel(const T *E, const int32_t *tok, int d, float *x) {
+  pdl_trigger();
+  pdl_wait();
   const T *src = E + (size_t)tok[blockIdx.x] * d;
   float *dst = x + (size_t)blockIdx.x * d;
   for (int i = threadIdx.x; i < d; i += blockDim.x) dst[i] = to_f<T>(src[i]);
 }
 void launch_embed(int dtype, const void *E, const int32_t *tok, int rows, int d, float *x, cudaStream_t s) {
   OURO_COUNT_LAUNCH();
-  if (dtype == OURO_BF16) embed_kernel<__nv_bfloat16><<<rows, 256, 0, s>>>((const __nv_bfloat16 *)E, tok, d, x);
-  else embed_kernel<float><<<rows, 256, 0, s>>>((const float *)E, tok, d, x);
+  if (dtype == OURO_BF16) launch_pdl(embed_kernel<__nv_bfloat16>, rows, 256, 0, s, (const __nv_bfloat16 *)E, tok, d, x);
+  else launch_pdl(embed_kernel<float>, rows, 256, 0, s, (const float *)E, tok, d, x);
 }
 
 // ----------------------------------------------------------------------------------- RMSNorm
 // out = g * x / sqrt(mean(x^2) + eps); one block per row, fixed reduction order.
 template <typename T>
 __global__ void rmsnorm_kernel(const float *x, const T *g, int d, float eps, T *out) {
+  pdl_trigger();
+  pdl_wait();
   const float *row = x + (size_t)blockIdx.x * d;
   float ss = 0.f;
   for (int i = threadIdx.x; i < d; i += blockDim.x) ss += row[i] * row[i];
@@ -95,8 +99,8 @@ __global__ void rmsnorm_kernel(const float *x, const T *g, int d, float eps, T *
 void launch_rmsnorm(int dtype, const float *x, const void *g, int rows, int d, float eps, void *out, cudaStream_t s) {
   OURO_COUNT_LAUNCH();
   if (dtype == OURO_BF16)
-    rmsnorm_kernel<__nv_bfloat16><<<rows, 256, 0, s>>>(x, (const __nv_bfloat16 *)g, d, eps, (__nv_bfloat16 *)out);
-  else rmsnorm_kernel<float><<<rows, 256, 0, s>>>(x, (const float *)g, d, eps, (float *)out);
+    launch_pdl(rmsnorm_kernel<__nv_bfloat16>, rows, 256, 0, s, x, (const __nv_bfloat16 *)g, d, eps, (__nv_bfloat16 *)out);
+  else launch_pdl(rmsnorm_kernel<float>, rows, 256, 0, s, x, (const float *)g, d, eps, (float *)out);
 }
 
 // -------------------------------------------------------------------------------- plain GEMM
@@ -192,6 +196,8 @@ void launch_gemm_swiglu_simple(int dtype, const void *X, const void *Wg, const v
 template <typename T>
 __global__ void rope_append_kernel(const float *qkv, const int32_t *pos, const float *cos_t, const float *sin_t,
                                    int H, int Hkv, int h, int L, size_t layer_off, T *q, T *k_cache, T *v_cache) {
+  pdl_trigger();
+  pdl_wait();
   int r = blockIdx.x, half = h >> 1, dq = H * h, dkv = Hkv * h;
   const float *row = qkv + (size_t)r * (dq + 2 * dkv);
   const float *c = cos_t + (size_t)pos[r] * half, *s = sin_t + (size_t)pos[r] * half;
@@ -213,12 +219,11 @@ void launch_rope_append(const ouro_model_desc &d, const float *qkv, const int32_
   OURO_COUNT_LAUNCH();
   size_t off = (size_t)layer * d.max_seq * d.n_kv_heads * d.head_dim;
   if (d.dtype == OURO_BF16)
-    rope_append_kernel<__nv_bfloat16><<<rows, 256, 0, s>>>(qkv, pos, cos_t, sin_t, d.n_heads, d.n_kv_heads, d.head_dim, L,
-                                                           off, (__nv_bfloat16 *)q, (__nv_bfloat16 *)k_cache,
-                                                           (__nv_bfloat16 *)v_cache);
+    launch_pdl(rope_append_kernel<__nv_bfloat16>, rows, 256, 0, s, qkv, pos, cos_t, sin_t, (int)d.n_heads, (int)d.n_kv_heads,
+               (int)d.head_dim, L, off, (__nv_bfloat16 *)q, (__nv_bfloat16 *)k_cache, (__nv_bfloat16 *)v_cache);
   else
-    rope_append_kernel<float><<<rows, 256, 0, s>>>(qkv, pos, cos_t, sin_t, d.n_heads, d.n_kv_heads, d.head_dim, L, off,
-                                                   (float *)q, (float *)k_cache, (float *)v_cache);
+    launch_pdl(rope_append_kernel<float>, rows, 256, 0, s, qkv, pos, cos_t, sin_t, (int)d.n_heads, (int)d.n_kv_heads,
+               (int)d.head_dim, L, off, (float *)q, (float *)k_cache, (float *)v_cache);
 }
 
 // ------------------------------------------------------------ candidate-masked attention (plain)

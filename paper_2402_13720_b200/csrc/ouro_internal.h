@@ -6,6 +6,7 @@
 #include <stdint.h>
 
 #include <string>
+#include <utility>
 #include <vector>
 
 #include "ouro.h"
@@ -14,6 +15,29 @@ typedef unsigned long long u64;
 
 extern unsigned long long g_ouro_launches;   // kernels launched by this library since it was loaded
 #define OURO_COUNT_LAUNCH() (++g_ouro_launches)
+
+// Programmatic dependent launch: a kernel launched with launch_pdl may start while its predecessor in the
+// stream is still draining.  Everything it does before pdl_wait() must be independent of earlier kernels
+// (set-up, prefetch of weights); pdl_wait() returns once the predecessor has completed and its writes are
+// visible.  pdl_trigger() lets the successor begin its own independent prologue.
+#ifdef __CUDACC__
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t s, Args &&...args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = s;
+  cudaLaunchAttribute at[1];
+  at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  at[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = at;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, std::forward<Args>(args)...);
+}
+#endif
 
 // Device-resident scalars of one decoding stream.
 struct DevState {
