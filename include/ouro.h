@@ -205,6 +205,26 @@ uint64_t ouro_kernel_launches(void);
 int ouro_profile_enable(ouro_ctx *ctx, int kernel_class);
 int ouro_profile_read(ouro_ctx *ctx, float *ms_total, int32_t *launches);
 
+/* (The paper has no counterpart to this call; it exists for deployment reasons only.)
+ * LM-head pass without any caller-provided workspace and without any allocation by the library: for callers
+ * that cannot allocate device memory - e.g. a server that gave all of it to its own arena at start-up, or a
+ * latency-critical loop that must avoid the device-wide synchronisation an allocation may cause.
+ *   x_dev        [rows, d_model] bf16, already normalised activations (device, 16-byte aligned)
+ *   lm_head_dev  [vocab, d_model] bf16, row-major (device, 16-byte aligned)
+ *   argmax_dev   [rows] int32 out: greedy token per row (ties -> smallest id)
+ *   logits_dev   [rows, vocab] fp32 out, or NULL
+ * Limits: 1 <= rows <= 128, d_model a multiple of 64, vocab a multiple of 8 and <= 65536; anything else returns
+ * OURO_EINVAL with a text in ouro_last_error(NULL).  The split-K scratch, counters and per-tile maxima live in a
+ * 5 MiB array inside the library image; every GPU that loads the library holds it until the process exits.
+ * The first call on each device resolves that array's device address and sizes the kernel's shared memory;
+ * make that first call outside any stream capture, with the device current.  All calls on a device share the
+ * array: two calls whose GPU work overlaps (different streams or threads) race on it - serialise them.
+ * The call enqueues on cuda_stream (a cudaStream_t, NULL = default), then synchronises that stream and returns
+ * OURO_ETIMEOUT if a bounded device-side wait gave up.  It runs on 32 SMs only (the scratch is sized per CTA), so
+ * it is slower than ouro_verify_forward's head pass; results agree with it to rounding (another split of K). */
+int ouro_lm_head_static(const void *x_dev, const void *lm_head_dev, int32_t rows, int32_t d_model, int32_t vocab,
+                        int32_t *argmax_dev, float *logits_dev, void *cuda_stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -77,6 +77,7 @@ _SIGNATURES = {
     "ouro_advance": (C.c_int, [C.c_void_p, C.c_int, C.c_int32]),
     "ouro_draft": (C.c_int, [C.c_void_p, C.c_void_p]),
     "ouro_kernel_launches": (C.c_uint64, []),
+    "ouro_lm_head_static": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p]),
     "ouro_profile_enable": (C.c_int, [C.c_void_p, C.c_int]),
     "ouro_profile_read": (C.c_int, [C.c_void_p, _F32P, _I32P]),
     "ouro_generate": (C.c_int, [C.c_void_p, _I32P, C.c_int32, C.c_int32, C.c_int32, _I32P, _I32P, C.POINTER(StatsC)]),
@@ -129,6 +130,24 @@ def params_c(p: synth.DecodeParams) -> ParamsC:
     flags = (OURO_HARVEST_MATCHED if p.harvest_matched else 0) | (OURO_HARVEST_CANDIDATES if p.harvest_candidates else 0) | \
             (OURO_HARVEST_ACCEPTED if p.harvest_accepted else 0) | (OURO_SEED_PROMPT if p.seed_prompt else 0)
     return ParamsC(p.gamma, p.beta, p.K, p.pool_sets, p.pool_ways, flags, p.eos_token)
+
+
+def lm_head_static(x: torch.Tensor, lm_head: torch.Tensor, want_logits: bool = False):
+    """LM-head pass for callers that cannot allocate: the library's own 5 MiB static array serves as scratch
+    (see ouro_lm_head_static in include/ouro.h).  x [rows, d] and lm_head [vocab, d] are bf16 CUDA tensors; the
+    outputs are allocated here by torch only because this is the Python convenience wrapper - the C call itself
+    allocates nothing.  Returns (argmax int32 [rows], logits fp32 [rows, vocab] or None)."""
+    assert x.is_cuda and lm_head.is_cuda and x.dtype == torch.bfloat16 and lm_head.dtype == torch.bfloat16
+    assert x.is_contiguous() and lm_head.is_contiguous() and x.shape[1] == lm_head.shape[1]
+    rows, d = x.shape
+    vocab = lm_head.shape[0]
+    argmax = torch.empty(rows, dtype=torch.int32, device=x.device)
+    logits = torch.empty((rows, vocab), dtype=torch.float32, device=x.device) if want_logits else None
+    with torch.cuda.device(x.device):
+        _check(lib().ouro_lm_head_static(x.data_ptr(), lm_head.data_ptr(), rows, d, vocab, argmax.data_ptr(),
+                                         logits.data_ptr() if want_logits else None,
+                                         torch.cuda.current_stream(x.device).cuda_stream))
+    return argmax, logits
 
 
 class _ModelMem:

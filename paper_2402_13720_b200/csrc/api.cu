@@ -40,6 +40,7 @@ extern "C" const char *ouro_strerror(int s) {
   }
   return "unknown status";
 }
+void ouro_set_global_error(const std::string &msg) { g_create_err = msg; }   // text for calls that have no context
 extern "C" const char *ouro_last_error(const ouro_ctx *c) { return c ? c->err.c_str() : g_create_err.c_str(); }
 
 // ---------------------------------------------------------------------------- workspace layout

@@ -21,6 +21,8 @@
 
 #include "ouro_internal.h"
 
+void ouro_set_global_error(const std::string &msg);   // api.cu
+
 namespace {
 
 constexpr int TILE_N = 128;       // weight rows per tile (MMA M)
@@ -828,6 +830,130 @@ int ouro_fast_head(ouro_ctx *c, int which, int rows, float *logits, int32_t *arg
   if (e != cudaSuccess) {
     c->err = std::string("tensor-core head launch: ") + cudaGetErrorString(e);
     return OURO_ECUDA;
+  }
+  return OURO_OK;
+}
+
+// ===================================================================================================
+// ouro_lm_head_static: the LM-head pass for callers that must not allocate.
+//
+// Some users of this library cannot give it a workspace: a serving process that handed all device memory to
+// its own arena at start-up (a later cudaMalloc simply fails), or a latency-critical loop that must not run
+// into the implicit device synchronisation an allocation can cause.  For them this one call keeps everything
+// the GEMM needs besides its inputs and outputs - the partial-tile slots of the split-K schedule, the tile
+// counters, the per-tile maxima and a status word - in a fixed array that is part of the library image.
+// Every GPU that loads the library carries these 5 MiB until the process exits.
+//
+// The array's name is only meaningful in device code.  Host code must ask the runtime for its device address
+// (cudaGetSymbolAddress) with the right device current; that is done once per device by the first call.
+// ===================================================================================================
+namespace {
+constexpr int NA_GRID = 32;                        // CTAs of the static-scratch launch (slots are per CTA)
+constexpr int NA_MAX_TILES = 512;                  // vocabulary <= 65536
+constexpr size_t NA_SLOT_BYTES = (size_t)NA_GRID * 2 * SLOT_FLOATS * sizeof(float);
+constexpr size_t NA_OFF_COUNTERS = NA_SLOT_BYTES;
+constexpr size_t NA_OFF_STATUS = NA_OFF_COUNTERS + NA_MAX_TILES * sizeof(int);
+constexpr size_t NA_OFF_TMAX = NA_OFF_STATUS + 256;
+constexpr size_t NA_OFF_TARG = NA_OFF_TMAX + (size_t)NA_MAX_TILES * OURO_MAX_ROWS * sizeof(float);
+constexpr size_t NA_BYTES = NA_OFF_TARG + (size_t)NA_MAX_TILES * OURO_MAX_ROWS * sizeof(int);
+static_assert(NA_BYTES <= (5u << 20), "the static scratch is documented as 5 MiB");
+constexpr int NA_MAX_DEVICES = 64;
+}  // namespace
+
+static __device__ __align__(256) unsigned char g_static_scratch[NA_BYTES];
+
+namespace {
+unsigned char *g_na_ptr[NA_MAX_DEVICES] = {};      // device address of g_static_scratch, per device
+int g_na_smem[NA_MAX_DEVICES] = {};
+
+// Once per device, with that device current: resolve the array's device address and size the kernel's
+// shared memory.  Returns OURO_OK or an error with a text for ouro_last_error(NULL).
+int na_setup(int dev) {
+  if (g_na_ptr[dev]) return OURO_OK;
+  void *ptr = nullptr;
+  cudaError_t e = cudaGetSymbolAddress(&ptr, g_static_scratch);
+  if (e != cudaSuccess || !ptr) {
+    ouro_set_global_error(std::string("cudaGetSymbolAddress(static scratch): ") + cudaGetErrorString(e));
+    return OURO_ECUDA;
+  }
+  int smem = 0;
+  if ((e = cudaDeviceGetAttribute(&smem, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev)) != cudaSuccess ||
+      (e = cudaFuncSetAttribute(gemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem)) != cudaSuccess) {
+    ouro_set_global_error(std::string("static-scratch set-up: ") + cudaGetErrorString(e));
+    return OURO_ECUDA;
+  }
+  if (!g_encode) {
+    void *fn = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess || !fn) {
+      ouro_set_global_error("cuTensorMapEncodeTiled unavailable");
+      return OURO_ECUDA;
+    }
+    g_encode = (EncodeTiledFn)fn;
+  }
+  g_na_smem[dev] = smem;
+  g_na_ptr[dev] = (unsigned char *)ptr;
+  return OURO_OK;
+}
+}  // namespace
+
+extern "C" int ouro_lm_head_static(const void *x_dev, const void *lm_head_dev, int32_t rows, int32_t d_model, int32_t vocab,
+                                   int32_t *argmax_dev, float *logits_dev, void *cuda_stream) {
+  if (!x_dev || !lm_head_dev || !argmax_dev) {
+    ouro_set_global_error("ouro_lm_head_static: null pointer");
+    return OURO_EINVAL;
+  }
+  if (rows < 1 || rows > OURO_MAX_ROWS || d_model < 64 || d_model % 64 != 0 || vocab < 8 || vocab % 8 != 0 ||
+      (vocab + TILE_N - 1) / TILE_N > NA_MAX_TILES || (((uintptr_t)x_dev | (uintptr_t)lm_head_dev) & 15)) {
+    ouro_set_global_error("ouro_lm_head_static: size beyond the static scratch (rows 1..128, d_model a multiple of 64, "
+                          "vocab a multiple of 8 and at most 65536) or pointers not 16-byte aligned");
+    return OURO_EINVAL;
+  }
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= NA_MAX_DEVICES) {
+    ouro_set_global_error("ouro_lm_head_static: no usable current device");
+    return OURO_ECUDA;
+  }
+  int rc = na_setup(dev);
+  if (rc != OURO_OK) return rc;
+  cudaStream_t s = (cudaStream_t)cuda_stream;
+  unsigned char *base = g_na_ptr[dev];
+  const int tiles = (vocab + TILE_N - 1) / TILE_N;
+  // the array keeps whatever the last call left: counters and status must start at zero
+  cudaError_t e = cudaMemsetAsync(base + NA_OFF_COUNTERS, 0, NA_OFF_TMAX - NA_OFF_COUNTERS, s);
+  GemmParams p{};
+  const int t_pad = (rows + 15) & ~15;
+  if (e != cudaSuccess || !make_map(&p.a[0], lm_head_dev, vocab, d_model, TILE_N) || !make_map(&p.b, x_dev, rows, d_model, t_pad)) {
+    ouro_set_global_error("ouro_lm_head_static: could not describe the operands to the copy engine");
+    return OURO_ECUDA;
+  }
+  p.a_tiles[0] = tiles; p.a_rows[0] = vocab; p.a_count = 1;
+  p.mode = MODE_HEAD;
+  p.tiles = tiles;
+  p.kb = d_model / BLOCK_K;
+  p.t_pad = t_pad;
+  p.rows = rows;
+  p.stages = stages_for(t_pad, g_na_smem[dev]);
+  p.out_f32 = logits_dev;
+  p.ldo = vocab;
+  p.tile_max = (float *)(base + NA_OFF_TMAX);
+  p.tile_arg = (int *)(base + NA_OFF_TARG);
+  p.scratch = (float *)base;
+  p.counters = (int *)(base + NA_OFF_COUNTERS);
+  p.status = (int *)(base + NA_OFF_STATUS);
+  const int total = tiles * p.kb;
+  gemm_tc_kernel<<<total < NA_GRID ? total : NA_GRID, THREADS, g_na_smem[dev], s>>>(p);
+  argmax_tiles_kernel<<<rows, 128, 0, s>>>(p.tile_max, p.tile_arg, tiles, argmax_dev);
+  int status = 0;
+  if ((e = cudaGetLastError()) != cudaSuccess ||
+      (e = cudaMemcpyAsync(&status, p.status, sizeof(int), cudaMemcpyDeviceToHost, s)) != cudaSuccess ||
+      (e = cudaStreamSynchronize(s)) != cudaSuccess) {
+    ouro_set_global_error(std::string("ouro_lm_head_static: ") + cudaGetErrorString(e));
+    return OURO_ECUDA;
+  }
+  if (status != 0) {
+    ouro_set_global_error("ouro_lm_head_static: a bounded device-side wait gave up");
+    return OURO_ETIMEOUT;
   }
   return OURO_OK;
 }
