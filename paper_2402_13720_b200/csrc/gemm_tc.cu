@@ -8,9 +8,11 @@
 //     are its N side; the fp32 accumulator [128 x T] lives in TMEM;
 //   * one persistent CTA per SM; the (tile, k-block) iteration space is cut into equal contiguous spans
 //     (stream-K), so every SM streams the same number of bytes whatever N and K are;
-//   * a span that covers only part of a tile's K range leaves a partial tile in scratch memory; the CTA that
-//     arrives last at the tile's counter adds the partials in ascending K order and runs the epilogue.
-//     Nobody waits for anybody, and the result does not depend on arrival order;
+//   * a span that covers only part of a tile's K range leaves a partial tile in scratch memory.  After its last
+//     MMA every contributor of a tile adds up a share of the tile's tokens (token t belongs to contributor
+//     t mod n) in ascending K order and runs the epilogue on them.  A CTA waits for the others' partials only
+//     after it has published all of its own, so the waits cannot form a cycle (and they are bounded); the
+//     result does not depend on arrival order;
 //   * warp 0 issues TMA loads into a ring of shared-memory stages (128-byte swizzle), warp 1 issues
 //     tcgen05.mma and releases stages with tcgen05.commit, warps 2-5 drain TMEM (double buffered) and run the
 //     epilogue: plain store, residual add, or SiLU(gate)*up for the stacked gate/up matrices.
@@ -55,7 +57,8 @@ struct GemmParams {
   float *tile_max;    // MODE_HEAD: [tiles][128] largest logit of each token inside the tile ...
   int *tile_arg;      //            ... and its vocabulary index (smallest index among equals)
   float *scratch;     // [grid][2][t][128] partial tiles
-  int *counters;      // [tiles], zero between launches
+  int *counters;      // [tiles] partial tiles published, zero between launches
+  int *done;          // [tiles] contributors that finished their share, zero between launches
   int *status;        // context status word
 };
 
@@ -123,6 +126,14 @@ __device__ __forceinline__ void tmem_ld16(uint32_t addr, float *v) {
 }
 __device__ __forceinline__ void fence_before_sync() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void fence_after_sync() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+// order-preserving map float -> uint32 (and back), so that integer max picks the largest float
+__device__ __forceinline__ uint32_t ordered_u32(float f) {
+  uint32_t u = __float_as_uint(f);
+  return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+__device__ __forceinline__ float ordered_f32(uint32_t u) {
+  return __uint_as_float((u & 0x80000000u) ? (u & 0x7fffffffu) : ~u);
+}
 __device__ __forceinline__ void epi_barrier() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
 
 struct Span {  // one piece of this CTA's work: k-blocks [kb0, kb1) of `tile`
@@ -209,7 +220,6 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_tc_kernel(const __grid_consta
   uint64_t *full = bars, *empty = bars + 16, *acc_full = bars + 32, *acc_empty = bars + 34;
   uint32_t *tmem_base_p = (uint32_t *)(bars + 36);
   volatile int *abort_flag = (volatile int *)(bars + 37);
-  int *last_flag = (int *)(bars + 38);
   volatile int *wait_flag = (volatile int *)(bars + 39);   // [2]: outcome of the epilogue's accumulator wait
 
   pdl_trigger();
@@ -330,8 +340,143 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_tc_kernel(const __grid_consta
     uint32_t item = 0;
     bool ok = true;
     float v[16];
+    int pend_tile[2], pend_n[2], pend_first[2], n_pend = 0;     // partial tiles this CTA contributed to (<= 2)
+
+    // Partial tiles: every contributor of a tile adds up a share of its tokens (token t belongs to contributor
+    // t mod n), in ascending K order.  Called once this CTA has published all its own partials, so waiting for
+    // the others cannot form a cycle; the wait is bounded all the same.  Loads of a batch of four tokens and four
+    // contributors are issued together, so a pass costs about one L2 round trip.
+    auto run_fixups = [&]() {
+      for (int k = 0; ok && k < n_pend; ++k) {
+        const int tile = pend_tile[k], n = pend_n[k], first = pend_first[k], my = (int)blockIdx.x - first;
+        if (et == 0) {
+          int seen = 0;
+          for (uint32_t i = 0; i < (1u << 22); ++i) {
+            asm volatile("ld.acquire.gpu.global.b32 %0, [%1];" : "=r"(seen) : "l"(p.counters + tile) : "memory");
+            if (seen >= n) break;
+            __nanosleep(20);
+          }
+          wait_flag[0] = seen >= n && !*abort_flag;
+        }
+        epi_barrier();
+        ok = wait_flag[0] != 0;
+        epi_barrier();
+        if (!ok) break;
+        __threadfence();
+        if (p.mode == MODE_SWIGLU) {
+          const int F = p.a_rows[0];
+          const int ng = et & 15, tg = et >> 4;                       // 4 features; tokens my + n*(tg + 8j)
+          const int feat = tile * 64 + 4 * ng;
+          for (int tb = my + n * tg; tb < p.rows; tb += n * 32) {
+            float4 g[4], u[4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) g[j] = u[j] = make_float4(0.f, 0.f, 0.f, 0.f);
+            for (int c0 = 0; c0 < n; c0 += 4) {
+              float4 tg4[4][4], tu4[4][4];
+#pragma unroll
+              for (int cc = 0; cc < 4; ++cc) {
+                const int owner = first + c0 + cc;
+                const float *src = p.scratch + ((size_t)owner * 2 + w.owner_slot(tile, owner)) * SLOT_FLOATS + 4 * ng;
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                  const int t = tb + j * n * 8;
+                  const bool in = c0 + cc < n && t < p.rows;
+                  tg4[cc][j] = in ? __ldcg((const float4 *)(src + (size_t)t * TILE_N)) : make_float4(0.f, 0.f, 0.f, 0.f);
+                  tu4[cc][j] = in ? __ldcg((const float4 *)(src + (size_t)t * TILE_N + 64)) : make_float4(0.f, 0.f, 0.f, 0.f);
+                }
+              }
+#pragma unroll
+              for (int cc = 0; cc < 4; ++cc)
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                  g[j].x += tg4[cc][j].x; g[j].y += tg4[cc][j].y; g[j].z += tg4[cc][j].z; g[j].w += tg4[cc][j].w;
+                  u[j].x += tu4[cc][j].x; u[j].y += tu4[cc][j].y; u[j].z += tu4[cc][j].z; u[j].w += tu4[cc][j].w;
+                }
+            }
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+              const int t = tb + j * n * 8;
+              if (t < p.rows && feat < F) {
+                __nv_bfloat162 lo = __floats2bfloat162_rn(g[j].x / (1.0f + __expf(-g[j].x)) * u[j].x, g[j].y / (1.0f + __expf(-g[j].y)) * u[j].y);
+                __nv_bfloat162 hi = __floats2bfloat162_rn(g[j].z / (1.0f + __expf(-g[j].z)) * u[j].z, g[j].w / (1.0f + __expf(-g[j].w)) * u[j].w);
+                *(uint2 *)(p.out_bf16 + (size_t)t * F + feat) = make_uint2(*(uint32_t *)&lo, *(uint32_t *)&hi);
+              }
+            }
+          }
+        } else {
+          int seg, row0, col0, valid;
+          locate(p, tile, seg, row0, col0, valid);
+          const int ng = et & 31, tg = et >> 5;                       // 4 columns; tokens my + n*(tg + 4j)
+          const int col = col0 + 4 * ng;
+          for (int tb = my + n * tg; tb < p.rows; tb += n * 16) {     // tokens are uniform inside a warp
+            float4 acc[4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) acc[j] = make_float4(0.f, 0.f, 0.f, 0.f);
+            for (int c0 = 0; c0 < n; c0 += 4) {
+              float4 tmp[4][4];
+#pragma unroll
+              for (int cc = 0; cc < 4; ++cc) {
+                const int owner = first + c0 + cc;
+                const float *src = p.scratch + ((size_t)owner * 2 + w.owner_slot(tile, owner)) * SLOT_FLOATS + 4 * ng;
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                  const int t = tb + j * n * 4;
+                  tmp[cc][j] = (c0 + cc < n && t < p.rows) ? __ldcg((const float4 *)(src + (size_t)t * TILE_N))
+                                                           : make_float4(0.f, 0.f, 0.f, 0.f);
+                }
+              }
+#pragma unroll
+              for (int cc = 0; cc < 4; ++cc)
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                  acc[j].x += tmp[cc][j].x; acc[j].y += tmp[cc][j].y; acc[j].z += tmp[cc][j].z; acc[j].w += tmp[cc][j].w;
+                }
+            }
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+              const int t = tb + j * n * 4;
+              if (t >= p.rows) continue;                              // uniform inside the warp
+              const float vals[4] = {acc[j].x, acc[j].y, acc[j].z, acc[j].w};
+              if (p.mode == MODE_HEAD) {                              // the warp's 32 lanes hold the tile's 128 columns
+                uint32_t bu = 0;
+                int bi = col;
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                  uint32_t uo = ordered_u32(vals[e]);
+                  if (4 * ng + e < valid && uo > bu) { bu = uo; bi = col + e; }
+                }
+                const uint32_t mx = __reduce_max_sync(0xffffffffu, bu);
+                const int src_lane = __ffs(__ballot_sync(0xffffffffu, bu == mx)) - 1;   // lowest lane = smallest index
+                bi = __shfl_sync(0xffffffffu, bi, src_lane);
+                if (lane == 0) {
+                  p.tile_max[(size_t)tile * OURO_MAX_ROWS + t] = ordered_f32(mx);
+                  p.tile_arg[(size_t)tile * OURO_MAX_ROWS + t] = bi;
+                }
+              }
+              if (p.out_f32) {
+                float *y = p.out_f32 + (size_t)t * p.ldo + col;
+#pragma unroll
+                for (int e = 0; e < 4; ++e)
+                  if (4 * ng + e < valid) y[e] = p.mode == MODE_RESIDUAL ? y[e] + vals[e] : vals[e];
+              }
+            }
+          }
+        }
+        epi_barrier();
+        if (et == 0) {                                                 // the last contributor to finish re-arms the tile
+          int d = atomicAdd(p.done + tile, 1);
+          if (d == n - 1) { p.counters[tile] = 0; p.done[tile] = 0; }
+        }
+      }
+      n_pend = 0;
+    };
+
     while (w.next(s)) {
       int a = item & 1;
+      // the stream-K spans come first: once the whole tiles start, this CTA has published all its partials and
+      // can add up its shares while the tensor cores work on the whole tile
+      if (s.n_contrib == 1 && n_pend > 0) run_fixups();
+      if (!ok) break;
       // one thread waits (bounded) and tells the others, so that all 128 leave the loop together
       if (et == 0) wait_flag[a] = mbar_wait(&acc_full[a], (item >> 1) & 1) && !*abort_flag;
       epi_barrier();
@@ -374,15 +519,10 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_tc_kernel(const __grid_consta
             if (p.mode == MODE_HEAD) {
 #pragma unroll
               for (int i = 0; i < 16; ++i) {
-                float bv = nl < valid ? v[i] : -INFINITY;
-                int bi = col0 + nl;
-#pragma unroll
-                for (int o = 16; o; o >>= 1) {
-                  float ov = __shfl_xor_sync(0xffffffffu, bv, o);
-                  int oi = __shfl_xor_sync(0xffffffffu, bi, o);
-                  if (ov > bv || (ov == bv && oi < bi)) { bv = ov; bi = oi; }
-                }
-                if (lane == 0) { xv[q * OURO_MAX_ROWS + t0 + i] = bv; xi[q * OURO_MAX_ROWS + t0 + i] = bi; }
+                const uint32_t bu = nl < valid ? ordered_u32(v[i]) : 0u;
+                const uint32_t mx = __reduce_max_sync(0xffffffffu, bu);
+                const int src_lane = __ffs(__ballot_sync(0xffffffffu, bu == mx)) - 1;   // smallest index among equals
+                if (lane == 0) { xv[q * OURO_MAX_ROWS + t0 + i] = ordered_f32(mx); xi[q * OURO_MAX_ROWS + t0 + i] = col0 + q * 32 + src_lane; }
               }
             }
           }
@@ -407,7 +547,7 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_tc_kernel(const __grid_consta
         __syncwarp();
         if (lane == 0) mbar_arrive(&acc_empty[a]);
       } else {
-        // partial tile: park it, and let the last arriver of the tile add everything up in K order
+        // partial tile: park it in this CTA's slot and announce it; the partials are added up after the loop
         float *mine = p.scratch + ((size_t)blockIdx.x * 2 + s.slot) * SLOT_FLOATS;
         for (int t0 = 0; t0 < p.t_pad; t0 += 16) {
           tmem_ld16(taddr + t0, v);
@@ -420,126 +560,15 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_tc_kernel(const __grid_consta
         if (lane == 0) mbar_arrive(&acc_empty[a]);
         __threadfence();
         epi_barrier();
-        if (et == 0) {
-          int old = atomicAdd(p.counters + s.tile, 1);
-          *last_flag = old == s.n_contrib - 1;
-          if (old == s.n_contrib - 1) p.counters[s.tile] = 0;     // ready for the next launch
-        }
-        epi_barrier();
-        const bool last = *last_flag != 0;
-        epi_barrier();
-        if (last) {
-          __threadfence();
-          // Sum the partial tiles in ascending K order.  Everything one thread needs for a batch of tokens
-          // is requested before the first add, so the pass runs at L2 bandwidth rather than L2 latency.
-          if (p.mode == MODE_SWIGLU) {
-            const int F = p.a_rows[0];
-            const int ng = et & 15, tg = et >> 4;                     // 4 features x tokens tg, tg+8, ..
-            const int feat = s.tile * 64 + 4 * ng;
-            for (int tb = 0; tb < p.rows; tb += 32) {
-              float4 g[4], u[4];
-#pragma unroll
-              for (int j = 0; j < 4; ++j) g[j] = u[j] = make_float4(0.f, 0.f, 0.f, 0.f);
-              for (int c0 = 0; c0 < s.n_contrib; c0 += 4) {
-                float4 tg4[4][4], tu4[4][4];
-#pragma unroll
-                for (int cc = 0; cc < 4; ++cc) {
-                  int owner = s.first_owner + c0 + cc;
-                  const float *src = p.scratch + ((size_t)owner * 2 + w.owner_slot(s.tile, owner)) * SLOT_FLOATS + 4 * ng;
-#pragma unroll
-                  for (int j = 0; j < 4; ++j) {
-                    int t = tb + tg + 8 * j;
-                    bool in = c0 + cc < s.n_contrib && t < p.rows;
-                    tg4[cc][j] = in ? __ldcg((const float4 *)(src + (size_t)t * TILE_N)) : make_float4(0.f, 0.f, 0.f, 0.f);
-                    tu4[cc][j] = in ? __ldcg((const float4 *)(src + (size_t)t * TILE_N + 64)) : make_float4(0.f, 0.f, 0.f, 0.f);
-                  }
-                }
-#pragma unroll
-                for (int cc = 0; cc < 4; ++cc)
-#pragma unroll
-                  for (int j = 0; j < 4; ++j) {
-                    g[j].x += tg4[cc][j].x; g[j].y += tg4[cc][j].y; g[j].z += tg4[cc][j].z; g[j].w += tg4[cc][j].w;
-                    u[j].x += tu4[cc][j].x; u[j].y += tu4[cc][j].y; u[j].z += tu4[cc][j].z; u[j].w += tu4[cc][j].w;
-                  }
-              }
-#pragma unroll
-              for (int j = 0; j < 4; ++j) {
-                int t = tb + tg + 8 * j;
-                if (t < p.rows && feat < F) {
-                  __nv_bfloat162 lo = __floats2bfloat162_rn(g[j].x / (1.0f + __expf(-g[j].x)) * u[j].x,
-                                                            g[j].y / (1.0f + __expf(-g[j].y)) * u[j].y);
-                  __nv_bfloat162 hi = __floats2bfloat162_rn(g[j].z / (1.0f + __expf(-g[j].z)) * u[j].z,
-                                                            g[j].w / (1.0f + __expf(-g[j].w)) * u[j].w);
-                  uint2 pk = make_uint2(*(uint32_t *)&lo, *(uint32_t *)&hi);
-                  *(uint2 *)(p.out_bf16 + (size_t)t * F + feat) = pk;
-                }
-              }
-            }
-          } else {
-            const int ng = et & 31, tg = et >> 5;                     // 4 columns x tokens tg, tg+4, ..
-            for (int tb = 0; tb < p.rows; tb += 32) {
-              float4 acc[8];
-#pragma unroll
-              for (int j = 0; j < 8; ++j) acc[j] = make_float4(0.f, 0.f, 0.f, 0.f);
-              for (int c0 = 0; c0 < s.n_contrib; c0 += 4) {
-                float4 tmp[4][8];
-#pragma unroll
-                for (int cc = 0; cc < 4; ++cc) {
-                  int owner = s.first_owner + c0 + cc;
-                  const float *src = p.scratch + ((size_t)owner * 2 + w.owner_slot(s.tile, owner)) * SLOT_FLOATS + 4 * ng;
-#pragma unroll
-                  for (int j = 0; j < 8; ++j) {
-                    int t = tb + tg + 4 * j;
-                    tmp[cc][j] = (c0 + cc < s.n_contrib && t < p.rows) ? __ldcg((const float4 *)(src + (size_t)t * TILE_N))
-                                                                       : make_float4(0.f, 0.f, 0.f, 0.f);
-                  }
-                }
-#pragma unroll
-                for (int cc = 0; cc < 4; ++cc)
-#pragma unroll
-                  for (int j = 0; j < 8; ++j) {
-                    acc[j].x += tmp[cc][j].x; acc[j].y += tmp[cc][j].y; acc[j].z += tmp[cc][j].z; acc[j].w += tmp[cc][j].w;
-                  }
-              }
-              const int col = col0 + 4 * ng;
-              if (p.mode == MODE_HEAD) {
-#pragma unroll
-                for (int j = 0; j < 8; ++j) {            // the 32 lanes of this warp cover the tile's 128 columns
-                  int t = tb + tg + 4 * j;
-                  float vals[4] = {acc[j].x, acc[j].y, acc[j].z, acc[j].w};
-                  float bv = -INFINITY;
-                  int bi = col;
-#pragma unroll
-                  for (int e = 0; e < 4; ++e)
-                    if (4 * ng + e < valid && vals[e] > bv) { bv = vals[e]; bi = col + e; }
-#pragma unroll
-                  for (int o = 16; o; o >>= 1) {
-                    float ov = __shfl_xor_sync(0xffffffffu, bv, o);
-                    int oi = __shfl_xor_sync(0xffffffffu, bi, o);
-                    if (ov > bv || (ov == bv && oi < bi)) { bv = ov; bi = oi; }
-                  }
-                  if (lane == 0 && t < p.rows) {
-                    p.tile_max[(size_t)s.tile * OURO_MAX_ROWS + t] = bv;
-                    p.tile_arg[(size_t)s.tile * OURO_MAX_ROWS + t] = bi;
-                  }
-                }
-              }
-#pragma unroll
-              for (int j = 0; j < 8; ++j) {
-                int t = tb + tg + 4 * j;
-                if (t >= p.rows || !p.out_f32) continue;
-                float *y = p.out_f32 + (size_t)t * p.ldo + col;
-                float vals[4] = {acc[j].x, acc[j].y, acc[j].z, acc[j].w};
-#pragma unroll
-                for (int e = 0; e < 4; ++e)
-                  if (4 * ng + e < valid) y[e] = p.mode == MODE_RESIDUAL ? y[e] + vals[e] : vals[e];
-              }
-            }
-          }
-        }
+        if (et == 0) atomicAdd(p.counters + s.tile, 1);
+        pend_tile[n_pend] = s.tile;
+        pend_n[n_pend] = s.n_contrib;
+        pend_first[n_pend] = s.first_owner;
+        ++n_pend;
       }
       ++item;
     }
+    run_fixups();
     if (!ok && et == 0) { *abort_flag = 1; atomicExch(p.status, 1); }
   }
   // ------------------------------------------------------------------ teardown
@@ -605,7 +634,7 @@ struct ouro_fast { FastState s; };
 size_t ouro_scratch_bytes(const ouro_model_desc *t, const ouro_model_desc *d) {
   size_t attn = attention_tc_scratch_bytes(*t);
   if (d && attention_tc_scratch_bytes(*d) > attn) attn = attention_tc_scratch_bytes(*d);
-  return slots_bytes() + MAX_TILES * sizeof(int) + 256 + 2 * tile_best_bytes() + attn;
+  return slots_bytes() + 2 * MAX_TILES * sizeof(int) + 256 + 2 * tile_best_bytes() + attn;
 }
 
 static bool shape_ok(const ouro_model_desc &d) {
@@ -639,10 +668,10 @@ int ouro_fast_setup(ouro_ctx *c) {
   f->s.smem_max = smem;
   f->s.slots = c->a.scratch;
   f->s.counters = (int *)((char *)c->a.scratch + slots_bytes());
-  f->s.tile_max = (float *)((char *)c->a.scratch + slots_bytes() + MAX_TILES * sizeof(int) + 256);
+  f->s.tile_max = (float *)((char *)c->a.scratch + slots_bytes() + 2 * MAX_TILES * sizeof(int) + 256);
   f->s.tile_arg = (int *)((char *)f->s.tile_max + tile_best_bytes());
   f->s.attn_part = (float *)((char *)f->s.tile_arg + tile_best_bytes());
-  if (cudaMemsetAsync(f->s.counters, 0, MAX_TILES * sizeof(int), c->stream) != cudaSuccess ||
+  if (cudaMemsetAsync(f->s.counters, 0, 2 * MAX_TILES * sizeof(int), c->stream) != cudaSuccess ||
       cudaFuncSetAttribute(gemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess ||
       attention_tc_setup() != OURO_OK) {
     delete f;
@@ -695,6 +724,7 @@ static void launch_gemm_tc(ouro_ctx *c, GemmParams &p, const CUtensorMap *xmaps,
   p.stages = stages_for(p.t_pad, s.smem_max);
   p.scratch = s.slots;
   p.counters = s.counters;
+  p.done = s.counters + MAX_TILES;
   p.status = &c->st->status;
   int total = p.tiles * p.kb;
   int grid = total < s.grid ? total : s.grid;
@@ -852,7 +882,7 @@ constexpr int NA_GRID = 32;                        // CTAs of the static-scratch
 constexpr int NA_MAX_TILES = 512;                  // vocabulary <= 65536
 constexpr size_t NA_SLOT_BYTES = (size_t)NA_GRID * 2 * SLOT_FLOATS * sizeof(float);
 constexpr size_t NA_OFF_COUNTERS = NA_SLOT_BYTES;
-constexpr size_t NA_OFF_STATUS = NA_OFF_COUNTERS + NA_MAX_TILES * sizeof(int);
+constexpr size_t NA_OFF_STATUS = NA_OFF_COUNTERS + 2 * NA_MAX_TILES * sizeof(int);   // published + finished counters
 constexpr size_t NA_OFF_TMAX = NA_OFF_STATUS + 256;
 constexpr size_t NA_OFF_TARG = NA_OFF_TMAX + (size_t)NA_MAX_TILES * OURO_MAX_ROWS * sizeof(float);
 constexpr size_t NA_BYTES = NA_OFF_TARG + (size_t)NA_MAX_TILES * OURO_MAX_ROWS * sizeof(int);
@@ -940,6 +970,7 @@ extern "C" int ouro_lm_head_static(const void *x_dev, const void *lm_head_dev, i
   p.tile_arg = (int *)(base + NA_OFF_TARG);
   p.scratch = (float *)base;
   p.counters = (int *)(base + NA_OFF_COUNTERS);
+  p.done = p.counters + NA_MAX_TILES;
   p.status = (int *)(base + NA_OFF_STATUS);
   const int total = tiles * p.kb;
   gemm_tc_kernel<<<total < NA_GRID ? total : NA_GRID, THREADS, g_na_smem[dev], s>>>(p);
