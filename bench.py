@@ -237,6 +237,62 @@ def workload_config(cache_len):
             "parallelism": "replicas"}
 
 
+def run_generate(args, device):
+    """End-to-end generation at batch 1: tokens/s of plain greedy decoding and of Ouroboros on the same GPU
+    kernels.  Drafts: "natural" = the draft model's own greedy tokens (random-init pairs agree at chance level);
+    "replay" = the target's recorded text with seeded substitutions and skips, standing in for a trained draft
+    model at three agreement levels (the draft model's forwards still run and are timed)."""
+    import dataclasses
+    from paper_2402_13720_b200 import binding, build
+    build.build()
+    T, D, P, R = synth.config(args.generate)
+    gen = args.gen_tokens or R["gen"]
+    need = R["n"] + gen + P.block_max + 8
+    T, D = dataclasses.replace(T, max_seq=max(T.max_seq, need)), dataclasses.replace(D, max_seq=max(D.max_seq, need))
+    wt = synth.model_weights(T, SEED, device=device)
+    wd = wt if args.generate == "C1" else synth.model_weights(D, SEED + 100, device=device)
+    eng = binding.Engine(T, wt, P, D, wd, device=device)
+    prompt = synth.prompt(SEED, T.vocab, R["n"], R["copy_frac"], *R["span"])
+    eng.generate_vanilla(prompt, min(gen, 16))                                    # warm-up
+    van, vs = eng.generate_vanilla(prompt, gen)
+    res = {"vanilla": {"tokens_per_s": len(van) / (vs["ms_total"] * 1e-3), "ms_per_token": vs["ms_total"] / len(van)}}
+    truth = np.concatenate([prompt, van, np.zeros(64, dtype=np.int32)])
+
+    def run(name, drafter):
+        eng.set_drafter(drafter)
+        out, st = eng.generate(prompt, gen)
+        eng.set_drafter(None)
+        res[name] = {"tokens_per_s": len(out) / (st["ms_total"] * 1e-3), "tokens_per_target_call": len(out) / st["target_calls"],
+                     "target_calls": st["target_calls"], "draft_calls": st["draft_calls"], "suffix_tokens": st["suffix_tokens"],
+                     "ms_target_per_call": st["ms_target"] / st["target_calls"],
+                     "ms_draft_per_step": st["ms_draft"] / st["target_calls"],
+                     "identical_to_vanilla": bool(np.array_equal(out, van))}
+
+    run("natural", None)
+    for name, (ps, pk) in {"replay_low": (0.30, 0.05), "replay_mid": (0.12, 0.03), "replay_high": (0.04, 0.01)}.items():
+        run(name, lambda seq, g, step, ps=ps, pk=pk: synth.corrupt_drafts(SEED + 7, truth, len(seq), g, T.vocab, ps, pk, step))
+    e = 2 if T.dtype == "bf16" else 4
+    wbytes = T.n_layers * T.layer_weight_elems() * e + T.vocab * T.d_model * e
+    peaks = {}
+    try:
+        peaks = json.load(open(os.path.join(ROOT, "MEASURED_PEAKS.json")))
+    except Exception:
+        pass
+    peak = peaks.get("hbm_gbs", 6650.0)
+    mid = res["replay_mid"]
+    line = {"metric": "generated_tokens_per_s_batch1", "value": mid["tokens_per_s"], "unit": "tokens/s", "n_gpus": 1,
+            "higher_is_better": True, "dtype": T.dtype, "data": "synthetic",
+            "config": {"workload": f"{args.generate}: prompt {R['n']}, generate {gen}, gamma {P.gamma}, beta {P.beta}, K {P.K}",
+                       "drafts": "replay_mid (seeded corruption of the target's own text: p_sub 0.12, p_skip 0.03)"},
+            "vs_vanilla": mid["tokens_per_s"] / res["vanilla"]["tokens_per_s"],
+            "vanilla_ceiling_tokens_per_s": peak * 1e9 / wbytes,
+            "verify_forward_gbs": wbytes / (mid["ms_target_per_call"] * 1e-3) / 1e9,
+            "verify_forward_frac_of_peak": wbytes / (mid["ms_target_per_call"] * 1e-3) / 1e9 / peak,
+            "results": res}
+    print(json.dumps(line))
+    eng.close()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -245,6 +301,10 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--cache-len", type=int, default=4096)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--generate", default=None, choices=["C1", "C3", "C4", "C5"],
+                    help="instead of the verify-step benchmark: whole generation on that configuration "
+                         "(vanilla greedy vs Ouroboros, natural and replayed drafts), one JSON line")
+    ap.add_argument("--gen-tokens", type=int, default=0, help="override the configuration's generation length")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -256,6 +316,8 @@ def main():
     from paper_2402_13720_b200 import binding, dist_util
     torch.cuda.set_device(local)
     device = f"cuda:{local}"
+    if args.generate:
+        return run_generate(args, device)
     group = dist_util.init(world, rank, "nccl") if world > 1 else None
     wl = GpuWorkload(device, args.cache_len)
     lib = binding.lib()
