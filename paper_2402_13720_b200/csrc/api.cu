@@ -371,6 +371,7 @@ extern "C" int ouro_profile_read(ouro_ctx *c, float *ms_total, int32_t *launches
 }
 
 // ----------------------------------------------------------------------------------- forward
+int ouro_fast_embed(ouro_ctx *c, int which, int rows);                     // embedding + first norm's inputs
 int ouro_fast_layer(ouro_ctx *c, int which, int layer, int rows);          // tensor-core layer; OURO_ESTATE = not available
 int ouro_fast_head(ouro_ctx *c, int which, int rows, float *logits, int32_t *argmax_dev);   // tensor-core LM head + argmax
 
@@ -384,7 +385,10 @@ static int forward(ouro_ctx *c, int which, int32_t *argmax_dev, float *logits_de
   cudaStream_t s = c->stream;
   Activations &a = c->a;
   ProfScope whole(c, OURO_PROF_FORWARD);
-  { ProfScope ps(c, OURO_PROF_EMBED); launch_embed(dt, M.embed, M.blk.tok, rows, d.d_model, a.x, s); }
+  if (ouro_fast_embed(c, which, rows) == OURO_ESTATE) {
+    ProfScope ps(c, OURO_PROF_EMBED);
+    launch_embed(dt, M.embed, M.blk.tok, rows, d.d_model, a.x, s);
+  }
   for (int l = 0; l < d.n_layers; ++l) {
     int rc = ouro_fast_layer(c, which, l, rows);
     if (rc == OURO_OK) continue;

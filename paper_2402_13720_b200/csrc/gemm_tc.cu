@@ -56,6 +56,15 @@ struct GemmParams {
   __nv_bfloat16 *out_bf16;  // MODE_SWIGLU: [rows, F]
   float *tile_max;    // MODE_HEAD: [tiles][128] largest logit of each token inside the tile ...
   int *tile_arg;      //            ... and its vocabulary index (smallest index among equals)
+  // RMSNorm folded into the GEMMs around it: g*x/rms(x) feeds a GEMM as bf16(g*x), and the per-token factor
+  // 1/rms(x) multiplies that GEMM's output instead.  The producer of x (a residual-add epilogue) leaves bf16(g*x)
+  // and, per 128-column tile, each token's sum of squares; the consumer adds the tile sums in order.
+  const __nv_bfloat16 *gain;  // MODE_RESIDUAL: gain of the norm that follows (NULL: plain residual add)
+  __nv_bfloat16 *xb;          // MODE_RESIDUAL: bf16(gain * x_new), [rows, ldo]
+  float *ss_out;              // MODE_RESIDUAL: [tiles][128] per-tile sums of squares of x_new
+  const float *ss_in;         // other modes: sums of squares of the activation rows (NULL: no scaling)
+  int ss_tiles;
+  float ss_inv_d, eps;
   float *scratch;     // [grid][2][t][128] partial tiles
   int *counters;      // [tiles] partial tiles published, zero between launches
   int *done;          // [tiles] contributors that finished their share, zero between launches
@@ -221,6 +230,7 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_tc_kernel(const __grid_consta
   uint32_t *tmem_base_p = (uint32_t *)(bars + 36);
   volatile int *abort_flag = (volatile int *)(bars + 37);
   volatile int *wait_flag = (volatile int *)(bars + 39);   // [2]: outcome of the epilogue's accumulator wait
+  float *rs = (float *)(bars + 48);                         // [128] per-token factor 1/rms of the consumed activations
 
   pdl_trigger();
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -396,6 +406,11 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_tc_kernel(const __grid_consta
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
               const int t = tb + j * n * 8;
+              if (t < p.rows) {
+                const float r = rs[t];
+                g[j].x *= r; g[j].y *= r; g[j].z *= r; g[j].w *= r;
+                u[j].x *= r; u[j].y *= r; u[j].z *= r; u[j].w *= r;
+              }
               if (t < p.rows && feat < F) {
                 __nv_bfloat162 lo = __floats2bfloat162_rn(g[j].x / (1.0f + __expf(-g[j].x)) * u[j].x, g[j].y / (1.0f + __expf(-g[j].y)) * u[j].y);
                 __nv_bfloat162 hi = __floats2bfloat162_rn(g[j].z / (1.0f + __expf(-g[j].z)) * u[j].z, g[j].w / (1.0f + __expf(-g[j].w)) * u[j].w);
@@ -436,7 +451,25 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_tc_kernel(const __grid_consta
             for (int j = 0; j < 4; ++j) {
               const int t = tb + j * n * 4;
               if (t >= p.rows) continue;                              // uniform inside the warp
-              const float vals[4] = {acc[j].x, acc[j].y, acc[j].z, acc[j].w};
+              if (p.mode == MODE_RESIDUAL && p.gain) {
+                float *y = p.out_f32 + (size_t)t * p.ldo + col;
+                const float add[4] = {acc[j].x, acc[j].y, acc[j].z, acc[j].w};
+                float sq = 0.f;
+#pragma unroll
+                for (int e = 0; e < 4; ++e)
+                  if (4 * ng + e < valid) {
+                    const float yn = y[e] + add[e];
+                    y[e] = yn;
+                    p.xb[(size_t)t * p.ldo + col + e] = __float2bfloat16_rn(__bfloat162float(p.gain[col + e]) * yn);
+                    sq += yn * yn;
+                  }
+#pragma unroll
+                for (int o = 16; o; o >>= 1) sq += __shfl_xor_sync(0xffffffffu, sq, o);
+                if (lane == 0) p.ss_out[(size_t)tile * OURO_MAX_ROWS + t] = sq;
+                continue;
+              }
+              const float r = rs[t];
+              const float vals[4] = {acc[j].x * r, acc[j].y * r, acc[j].z * r, acc[j].w * r};
               if (p.mode == MODE_HEAD) {                              // the warp's 32 lanes hold the tile's 128 columns
                 uint32_t bu = 0;
                 int bi = col;
@@ -471,6 +504,17 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_tc_kernel(const __grid_consta
       n_pend = 0;
     };
 
+    if (et < OURO_MAX_ROWS) {
+      float r = 1.0f;
+      if (p.ss_in && et < p.rows) {
+        float sum = 0.f;
+        for (int i = 0; i < p.ss_tiles; ++i) sum += p.ss_in[(size_t)i * OURO_MAX_ROWS + et];
+        r = 1.0f / sqrtf(sum * p.ss_inv_d + p.eps);
+      }
+      rs[et] = r;
+    }
+    epi_barrier();
+
     while (w.next(s)) {
       int a = item & 1;
       // the stream-K spans come first: once the whole tiles start, this CTA has published all its partials and
@@ -493,9 +537,11 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_tc_kernel(const __grid_consta
           const int feat = s.tile * 64 + (nl & 63);
           for (int t0 = 0; t0 < p.t_pad; t0 += 16) {
             tmem_ld16(taddr + t0, v);
+#pragma unroll
+            for (int i = 0; i < 16; ++i) v[i] *= rs[t0 + i];
             if (nl >= 64) {
 #pragma unroll
-              for (int i = 0; i < 16; ++i) xchg[(nl - 64) * OURO_MAX_ROWS + t0 + i] = v[i];
+              for (int i = 0; i < 16; ++i) xchg[(t0 + i) * 64 + (nl - 64)] = v[i];
             }
             epi_barrier();
             if (nl < 64 && feat < F) {
@@ -503,7 +549,7 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_tc_kernel(const __grid_consta
               for (int i = 0; i < 16; ++i) {
                 int t = t0 + i;
                 if (t < p.rows) {
-                  float g = v[i], u = xchg[nl * OURO_MAX_ROWS + t];
+                  float g = v[i], u = xchg[t * 64 + nl];
                   p.out_bf16[(size_t)t * F + feat] = __float2bfloat16_rn(g / (1.0f + __expf(-g)) * u);
                 }
               }
@@ -515,6 +561,28 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_tc_kernel(const __grid_consta
           int *xi = (int *)(xchg + 4 * OURO_MAX_ROWS);        //                         and its index
           for (int t0 = 0; t0 < p.t_pad; t0 += 16) {
             tmem_ld16(taddr + t0, v);
+            if (p.mode == MODE_RESIDUAL && p.gain) {
+              // new residual stream, its bf16(gain * x) image for the next GEMM, and this tile's sums of squares
+              const float gcol = nl < valid ? __bfloat162float(p.gain[col0 + nl]) : 0.f;
+#pragma unroll
+              for (int i = 0; i < 16; ++i) {
+                const int t = t0 + i;
+                float y = 0.f;
+                if (t < p.rows && nl < valid) {
+                  float *yp = p.out_f32 + (size_t)t * p.ldo + col0 + nl;
+                  y = *yp + v[i];
+                  *yp = y;
+                  p.xb[(size_t)t * p.ldo + col0 + nl] = __float2bfloat16_rn(gcol * y);
+                }
+                float sq = y * y;
+#pragma unroll
+                for (int o = 16; o; o >>= 1) sq += __shfl_xor_sync(0xffffffffu, sq, o);
+                if (lane == 0) xv[q * OURO_MAX_ROWS + t] = sq;
+              }
+              continue;
+            }
+#pragma unroll
+            for (int i = 0; i < 16; ++i) v[i] *= rs[t0 + i];
             store_chunk(p, col0 + nl, nl < valid, t0, v);
             if (p.mode == MODE_HEAD) {
 #pragma unroll
@@ -525,6 +593,13 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_tc_kernel(const __grid_consta
                 if (lane == 0) { xv[q * OURO_MAX_ROWS + t0 + i] = ordered_f32(mx); xi[q * OURO_MAX_ROWS + t0 + i] = col0 + q * 32 + src_lane; }
               }
             }
+          }
+          if (p.mode == MODE_RESIDUAL && p.gain) {
+            epi_barrier();
+            if (et < p.rows)
+              p.ss_out[(size_t)s.tile * OURO_MAX_ROWS + et] =
+                  ((xv[et] + xv[OURO_MAX_ROWS + et]) + xv[2 * OURO_MAX_ROWS + et]) + xv[3 * OURO_MAX_ROWS + et];
+            epi_barrier();
           }
           if (p.mode == MODE_HEAD) {
             epi_barrier();
@@ -614,15 +689,18 @@ struct FastState {
   float *attn_part = nullptr;   // per-chunk softmax pieces of the split attention
   float *tile_max = nullptr;    // LM head: per-tile best logit and index of every token
   int *tile_arg = nullptr;
+  float *ss = nullptr;          // per-tile sums of squares of the residual stream (RMSNorm folded into the GEMMs)
 };
 constexpr int MAX_TILES = 4096;
 
 size_t slots_bytes() { return (size_t)MAX_GRID * 2 * SLOT_FLOATS * sizeof(float); }
 size_t tile_best_bytes() { return (size_t)MAX_TILES * OURO_MAX_ROWS * 4; }
+constexpr int MAX_SS_TILES = 64;           // d_model <= 8192
+size_t ss_bytes() { return (size_t)MAX_SS_TILES * OURO_MAX_ROWS * sizeof(float); }
 
 int stages_for(int t_pad, int smem_max) {
   int stage = A_BYTES + t_pad * BLOCK_K * 2;
-  int fixed = 1024 + 64 * OURO_MAX_ROWS * 4 + 512;   // alignment slack, SwiGLU exchange buffer, barriers and flags
+  int fixed = 1024 + 64 * OURO_MAX_ROWS * 4 + 1024;  // alignment slack, exchange buffer, barriers, flags, per-token factors
   int s = (smem_max - fixed) / stage;
   return s > 12 ? 12 : s;
 }
@@ -634,12 +712,12 @@ struct ouro_fast { FastState s; };
 size_t ouro_scratch_bytes(const ouro_model_desc *t, const ouro_model_desc *d) {
   size_t attn = attention_tc_scratch_bytes(*t);
   if (d && attention_tc_scratch_bytes(*d) > attn) attn = attention_tc_scratch_bytes(*d);
-  return slots_bytes() + 2 * MAX_TILES * sizeof(int) + 256 + 2 * tile_best_bytes() + attn;
+  return slots_bytes() + 2 * MAX_TILES * sizeof(int) + 256 + 2 * tile_best_bytes() + ss_bytes() + attn;
 }
 
 static bool shape_ok(const ouro_model_desc &d) {
   int dq = d.n_heads * d.head_dim;
-  return d.dtype == OURO_BF16 && d.d_model % 64 == 0 && dq % 64 == 0 && d.d_ffn % 64 == 0 && d.vocab % 8 == 0 &&
+  return d.dtype == OURO_BF16 && d.d_model % 64 == 0 && d.d_model <= MAX_SS_TILES * TILE_N && dq % 64 == 0 && d.d_ffn % 64 == 0 && d.vocab % 8 == 0 &&
          (d.vocab + TILE_N - 1) / TILE_N <= MAX_TILES && (2 * d.d_ffn + TILE_N - 1) / TILE_N <= MAX_TILES;
 }
 
@@ -670,7 +748,8 @@ int ouro_fast_setup(ouro_ctx *c) {
   f->s.counters = (int *)((char *)c->a.scratch + slots_bytes());
   f->s.tile_max = (float *)((char *)c->a.scratch + slots_bytes() + 2 * MAX_TILES * sizeof(int) + 256);
   f->s.tile_arg = (int *)((char *)f->s.tile_max + tile_best_bytes());
-  f->s.attn_part = (float *)((char *)f->s.tile_arg + tile_best_bytes());
+  f->s.ss = (float *)((char *)f->s.tile_arg + tile_best_bytes());
+  f->s.attn_part = (float *)((char *)f->s.ss + ss_bytes());
   if (cudaMemsetAsync(f->s.counters, 0, 2 * MAX_TILES * sizeof(int), c->stream) != cudaSuccess ||
       cudaFuncSetAttribute(gemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess ||
       attention_tc_setup() != OURO_OK) {
@@ -731,6 +810,45 @@ static void launch_gemm_tc(ouro_ctx *c, GemmParams &p, const CUtensorMap *xmaps,
   launch_pdl(gemm_tc_kernel, grid, THREADS, (size_t)s.smem_max, c->stream, p);
 }
 
+// Embedding rows into the residual stream, plus what the first norm's consumer needs: bf16(gain * x) and each
+// row's sum of squares (kept in tile 0 of the per-tile array, the other tiles zero).
+__global__ void embed_norm_kernel(const __nv_bfloat16 *E, const int32_t *tok, int d, const __nv_bfloat16 *gain, float *x,
+                                  __nv_bfloat16 *xb, float *ss, int ss_tiles) {
+  pdl_trigger();
+  pdl_wait();
+  const int r = blockIdx.x;
+  const __nv_bfloat16 *src = E + (size_t)tok[r] * d;
+  float sq = 0.f;
+  for (int i = threadIdx.x; i < d; i += blockDim.x) {
+    float v = __bfloat162float(src[i]);
+    x[(size_t)r * d + i] = v;
+    xb[(size_t)r * d + i] = __float2bfloat16_rn(__bfloat162float(gain[i]) * v);
+    sq += v * v;
+  }
+  __shared__ float part[8];
+#pragma unroll
+  for (int o = 16; o; o >>= 1) sq += __shfl_xor_sync(0xffffffffu, sq, o);
+  if ((threadIdx.x & 31) == 0) part[threadIdx.x >> 5] = sq;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    float tot = 0.f;
+    for (int w = 0; w < (int)(blockDim.x >> 5); ++w) tot += part[w];
+    ss[r] = tot;
+  }
+  for (int i = 1 + threadIdx.x; i < ss_tiles; i += blockDim.x) ss[(size_t)i * OURO_MAX_ROWS + r] = 0.f;
+}
+
+int ouro_fast_embed(ouro_ctx *c, int which, int rows) {
+  if (!c->fast || !c->fast->s.m[which].ok) return OURO_ESTATE;
+  ModelRt &M = c->m[which];
+  const ouro_model_desc &d = M.d;
+  ProfScope ps(c, OURO_PROF_EMBED);
+  OURO_COUNT_LAUNCH();
+  launch_pdl(embed_norm_kernel, rows, 256, 0, c->stream, (const __nv_bfloat16 *)M.embed, (const int32_t *)M.blk.tok, (int)d.d_model,
+             (const __nv_bfloat16 *)M.attn_norm[0], c->a.x, (__nv_bfloat16 *)c->a.xn, c->fast->s.ss, (int)((d.d_model + TILE_N - 1) / TILE_N));
+  return OURO_OK;
+}
+
 // One decoder layer with the tensor-core GEMMs; OURO_ESTATE when the model does not qualify.
 int ouro_fast_layer(ouro_ctx *c, int which, int l, int rows) {
   if (!c->fast || !c->fast->s.m[which].ok) return OURO_ESTATE;
@@ -742,7 +860,11 @@ int ouro_fast_layer(ouro_ctx *c, int which, int l, int rows) {
   cudaStream_t s = c->stream;
   LayerMaps &lm = fm.layers[l];
   auto tiles = [](int n) { return (n + TILE_N - 1) / TILE_N; };
-  { ProfScope ps(c, OURO_PROF_NORM); launch_rmsnorm(OURO_BF16, a.x, M.attn_norm[l], rows, d.d_model, d.rms_eps, a.xn, s); }
+  // a.xn holds bf16(attn_norm * x) and ss the sums of squares, left by the embedding or the previous layer's down GEMM
+  float *ss = c->fast->s.ss;
+  const int ss_tiles = tiles(d.d_model);
+  auto consume = [&](GemmParams &p) { p.ss_in = ss; p.ss_tiles = ss_tiles; p.ss_inv_d = 1.0f / (float)d.d_model; p.eps = d.rms_eps; };
+  auto produce = [&](GemmParams &p, const void *gain) { p.gain = (const __nv_bfloat16 *)gain; p.xb = (__nv_bfloat16 *)a.xn; p.ss_out = ss; };
   {
     ProfScope ps(c, OURO_PROF_QKV);
     GemmParams p{};
@@ -754,6 +876,7 @@ int ouro_fast_layer(ouro_ctx *c, int which, int l, int rows) {
     p.tiles = p.a_tiles[0] + p.a_tiles[1] + p.a_tiles[2];
     p.out_f32 = a.qkv;
     p.ldo = dq + 2 * dkv;
+    consume(p);
     launch_gemm_tc(c, p, fm.x_d, d.d_model, rows);
   }
   { ProfScope ps(c, OURO_PROF_ROPE); launch_rope_append(d, a.qkv, M.blk.pos, M.rope_cos, M.rope_sin, rows, M.L, l, a.q, M.k_cache, M.v_cache, s); }
@@ -772,9 +895,9 @@ int ouro_fast_layer(ouro_ctx *c, int which, int l, int rows) {
     p.tiles = p.a_tiles[0];
     p.out_f32 = a.x;
     p.ldo = d.d_model;
+    produce(p, M.ffn_norm[l]);
     launch_gemm_tc(c, p, fm.x_q, dq, rows);
   }
-  { ProfScope ps(c, OURO_PROF_NORM); launch_rmsnorm(OURO_BF16, a.x, M.ffn_norm[l], rows, d.d_model, d.rms_eps, a.xn, s); }
   {
     ProfScope ps(c, OURO_PROF_GATEUP);
     GemmParams p{};
@@ -782,6 +905,7 @@ int ouro_fast_layer(ouro_ctx *c, int which, int l, int rows) {
     p.mode = MODE_SWIGLU;
     p.tiles = (d.d_ffn + 63) / 64;
     p.out_bf16 = (__nv_bfloat16 *)a.act;
+    consume(p);
     launch_gemm_tc(c, p, fm.x_d, d.d_model, rows);
   }
   {
@@ -792,6 +916,7 @@ int ouro_fast_layer(ouro_ctx *c, int which, int l, int rows) {
     p.tiles = p.a_tiles[0];
     p.out_f32 = a.x;
     p.ldo = d.d_model;
+    produce(p, l + 1 < d.n_layers ? M.attn_norm[l + 1] : M.final_norm);
     launch_gemm_tc(c, p, fm.x_f, d.d_ffn, rows);
   }
   cudaError_t e = cudaGetLastError();
@@ -837,7 +962,6 @@ int ouro_fast_head(ouro_ctx *c, int which, int rows, float *logits, int32_t *arg
   ModelRt &M = c->m[which];
   FastModel &fm = c->fast->s.m[which];
   const ouro_model_desc &d = M.d;
-  { ProfScope ps(c, OURO_PROF_NORM); launch_rmsnorm(OURO_BF16, c->a.x, M.final_norm, rows, d.d_model, d.rms_eps, c->a.xn, c->stream); }
   {
     ProfScope ps(c, OURO_PROF_HEAD);
     GemmParams p{};
@@ -848,6 +972,7 @@ int ouro_fast_head(ouro_ctx *c, int which, int rows, float *logits, int32_t *arg
     p.ldo = d.vocab;
     p.tile_max = c->fast->s.tile_max;
     p.tile_arg = c->fast->s.tile_arg;
+    p.ss_in = c->fast->s.ss; p.ss_tiles = (d.d_model + TILE_N - 1) / TILE_N; p.ss_inv_d = 1.0f / (float)d.d_model; p.eps = d.rms_eps;
     launch_gemm_tc(c, p, fm.x_d, d.d_model, rows);
   }
   {
