@@ -37,7 +37,8 @@ constexpr uint32_t SPIN_LIMIT = 1u << 24;
 constexpr unsigned long long HINT_EVICT_FIRST = 0x12F0000000000000ull;
 constexpr unsigned long long HINT_EVICT_LAST = 0x14F0000000000000ull;
 
-enum { MODE_STORE = 0, MODE_RESIDUAL = 1, MODE_SWIGLU = 2, MODE_HEAD = 3 };   // HEAD: per-tile row maxima (+ optional logits)
+enum { MODE_STORE = 0, MODE_RESIDUAL = 1, MODE_SWIGLU = 2, MODE_HEAD = 3, MODE_QKV = 4 };
+// HEAD: per-tile row maxima (+ optional logits).  QKV: rotary positions on q and k, q to its buffer, k and v appended to the cache.
 
 struct GemmParams {
   CUtensorMap a[3];   // weight matrices stacked along the output dimension (q|k|v), or gate and up
@@ -59,6 +60,12 @@ struct GemmParams {
   // RMSNorm folded into the GEMMs around it: g*x/rms(x) feeds a GEMM as bf16(g*x), and the per-token factor
   // 1/rms(x) multiplies that GEMM's output instead.  The producer of x (a residual-add epilogue) leaves bf16(g*x)
   // and, per 128-column tile, each token's sum of squares; the consumer adds the tile sums in order.
+  // MODE_QKV: stacked q|k|v tiles hold whole heads (head_dim 64 or 128); pairs (i, i + head_dim/2) are rotated by
+  // the row's position; q goes to q_out [rows, dq], k and v to cache slots L + row of this layer
+  const int32_t *pos;
+  const float *cos_t, *sin_t;   // [max_seq, head_dim/2]
+  __nv_bfloat16 *q_out, *k_out, *v_out;
+  int head_dim, dq, dkv, L;
   const __nv_bfloat16 *gain;  // MODE_RESIDUAL: gain of the norm that follows (NULL: plain residual add)
   __nv_bfloat16 *xb;          // MODE_RESIDUAL: bf16(gain * x_new), [rows, ldo]
   float *ss_out;              // MODE_RESIDUAL: [tiles][128] per-tile sums of squares of x_new
@@ -470,6 +477,28 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_tc_kernel(const __grid_consta
               }
               const float r = rs[t];
               const float vals[4] = {acc[j].x * r, acc[j].y * r, acc[j].z * r, acc[j].w * r};
+              if (p.mode == MODE_QKV) {
+                const int cm = row0 + 4 * ng;                    // first of this thread's 4 columns inside q, k or v
+                const int half = p.head_dim >> 1;
+                float other[4];
+#pragma unroll
+                for (int e = 0; e < 4; ++e) other[e] = __shfl_xor_sync(0xffffffffu, vals[e], half >> 2);
+                const bool upper = (cm & half) != 0;
+                const size_t ti = (size_t)p.pos[t] * half + (cm & (half - 1));
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                  if (4 * ng + e >= valid) continue;
+                  if (seg == 2) {
+                    p.v_out[(size_t)(p.L + t) * p.dkv + cm + e] = __float2bfloat16_rn(vals[e]);
+                  } else {
+                    const float cs = p.cos_t[ti + e], sn = p.sin_t[ti + e];
+                    const float rv = upper ? vals[e] * cs + other[e] * sn : vals[e] * cs - other[e] * sn;
+                    if (seg == 0) p.q_out[(size_t)t * p.dq + cm + e] = __float2bfloat16_rn(rv);
+                    else p.k_out[(size_t)(p.L + t) * p.dkv + cm + e] = __float2bfloat16_rn(rv);
+                  }
+                }
+                continue;
+              }
               if (p.mode == MODE_HEAD) {                              // the warp's 32 lanes hold the tile's 128 columns
                 uint32_t bu = 0;
                 int bi = col;
@@ -583,6 +612,37 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_tc_kernel(const __grid_consta
             }
 #pragma unroll
             for (int i = 0; i < 16; ++i) v[i] *= rs[t0 + i];
+            if (p.mode == MODE_QKV) {
+              const int cm = row0 + nl;                          // column inside q, k or v
+              if (seg == 2) {
+                if (nl < valid)
+#pragma unroll
+                  for (int i = 0; i < 16; ++i)
+                    if (t0 + i < p.rows) p.v_out[(size_t)(p.L + t0 + i) * p.dkv + cm] = __float2bfloat16_rn(v[i]);
+              } else {
+                const int half = p.head_dim >> 1, ih = cm & (half - 1);
+                const bool upper = (cm & half) != 0;
+#pragma unroll
+                for (int i = 0; i < 16; ++i) xchg[i * TILE_N + nl] = v[i];
+                epi_barrier();
+                if (nl < valid) {
+#pragma unroll
+                  for (int i = 0; i < 16; ++i) {
+                    const int t = t0 + i;
+                    if (t < p.rows) {
+                      const float other = xchg[i * TILE_N + (nl ^ half)];
+                      const size_t ti = (size_t)p.pos[t] * half + ih;
+                      const float cs = p.cos_t[ti], sn = p.sin_t[ti];
+                      const float r = upper ? v[i] * cs + other * sn : v[i] * cs - other * sn;
+                      if (seg == 0) p.q_out[(size_t)t * p.dq + cm] = __float2bfloat16_rn(r);
+                      else p.k_out[(size_t)(p.L + t) * p.dkv + cm] = __float2bfloat16_rn(r);
+                    }
+                  }
+                }
+                epi_barrier();
+              }
+              continue;
+            }
             store_chunk(p, col0 + nl, nl < valid, t0, v);
             if (p.mode == MODE_HEAD) {
 #pragma unroll
@@ -872,14 +932,28 @@ int ouro_fast_layer(ouro_ctx *c, int which, int l, int rows) {
     p.a_tiles[0] = tiles(dq); p.a_tiles[1] = tiles(dkv); p.a_tiles[2] = tiles(dkv);
     p.a_rows[0] = dq; p.a_rows[1] = dkv; p.a_rows[2] = dkv;
     p.a_count = 3;
-    p.mode = MODE_STORE;
     p.tiles = p.a_tiles[0] + p.a_tiles[1] + p.a_tiles[2];
-    p.out_f32 = a.qkv;
-    p.ldo = dq + 2 * dkv;
     consume(p);
+    const bool fused_rope = d.head_dim == 64 || d.head_dim == 128;   // tiles then hold whole heads
+    if (fused_rope) {
+      const size_t off = (size_t)l * d.max_seq * dkv;
+      p.mode = MODE_QKV;
+      p.pos = M.blk.pos; p.cos_t = M.rope_cos; p.sin_t = M.rope_sin;
+      p.q_out = (__nv_bfloat16 *)a.q;
+      p.k_out = (__nv_bfloat16 *)M.k_cache + off;
+      p.v_out = (__nv_bfloat16 *)M.v_cache + off;
+      p.head_dim = d.head_dim; p.dq = dq; p.dkv = dkv; p.L = M.L;
+    } else {
+      p.mode = MODE_STORE;
+      p.out_f32 = a.qkv;
+      p.ldo = dq + 2 * dkv;
+    }
     launch_gemm_tc(c, p, fm.x_d, d.d_model, rows);
+    if (!fused_rope) {
+      ProfScope pr(c, OURO_PROF_ROPE);
+      launch_rope_append(d, a.qkv, M.blk.pos, M.rope_cos, M.rope_sin, rows, M.L, l, a.q, M.k_cache, M.v_cache, s);
+    }
   }
-  { ProfScope ps(c, OURO_PROF_ROPE); launch_rope_append(d, a.qkv, M.blk.pos, M.rope_cos, M.rope_sin, rows, M.L, l, a.q, M.k_cache, M.v_cache, s); }
   {
     ProfScope ps(c, OURO_PROF_ATTENTION);
     if (attention_tc_supported(d))
