@@ -271,6 +271,21 @@ def run_generate(args, device):
     run("natural", None)
     for name, (ps, pk) in {"replay_low": (0.30, 0.05), "replay_mid": (0.12, 0.03), "replay_high": (0.04, 0.01)}.items():
         run(name, lambda seq, g, step, ps=ps, pk=pk: synth.corrupt_drafts(SEED + 7, truth, len(seq), g, T.vocab, ps, pk, step))
+
+    # A random-init target does not repeat its prompt, so the pool (filled from the prompt and the accepted text)
+    # rarely holds a phrase that starts with the draft's last token.  The paper's main phrase source, n-grams
+    # produced during the draft model's forwards (Section 3.1), is not specified there; this stand-in feeds the pool
+    # each step with K phrases that continue the draft: the recorded text after it, corrupted like the drafts.
+    def with_phrases(seq, g, step):
+        d = synth.corrupt_drafts(SEED + 7, truth, len(seq), g, T.vocab, 0.12, 0.03, step)
+        grams = np.empty((P.K, P.beta), dtype=np.int32)
+        for j in range(P.K):
+            grams[j, 0] = d[-1]
+            grams[j, 1:] = synth.corrupt_drafts(SEED + 11 + j, truth, len(seq) + g, P.S, T.vocab, 0.08 * (j + 1), 0.0, step)
+        eng.phrase_update(grams[::-1])                      # the least corrupted phrase is inserted last = looked up first
+        return d
+
+    run("replay_mid_phrases", with_phrases)
     e = 2 if T.dtype == "bf16" else 4
     wbytes = T.n_layers * T.layer_weight_elems() * e + T.vocab * T.d_model * e
     peaks = {}
@@ -288,6 +303,7 @@ def run_generate(args, device):
             "vanilla_ceiling_tokens_per_s": peak * 1e9 / wbytes,
             "verify_forward_gbs": wbytes / (mid["ms_target_per_call"] * 1e-3) / 1e9,
             "verify_forward_frac_of_peak": wbytes / (mid["ms_target_per_call"] * 1e-3) / 1e9 / peak,
+            "with_phrases_vs_vanilla": res["replay_mid_phrases"]["tokens_per_s"] / res["vanilla"]["tokens_per_s"],
             "results": res}
     print(json.dumps(line))
     eng.close()

@@ -6,7 +6,8 @@
 // and the kernel maps "virtual positions" 0..n_vis-1 to cache slots on the fly.
 //
 // Work split.  Keys are cut by virtual position into aligned spans of 512; one CTA handles one (kv head, span)
-// for all query rows and all query heads of the group, so every cached byte is read from HBM once.  The CTA
+// for up to 64 query rows (rows x query heads of the group; further rows go to further CTAs, which find the same
+// keys in L2), so every cached byte is read from HBM once.  The CTA
 // walks its span in chunks of 128 keys: K and V rows of the next chunk stream into a second shared-memory
 // buffer (cp.async) while the current one is used.  Per chunk: the 8 warps split the keys for S = Q K^T
 // (mma.sync), agree on each row's chunk maximum through shared memory, write P = exp2(S - max) as bf16 to shared
@@ -132,8 +133,9 @@ __global__ void __launch_bounds__(THREADS) attn_span_kernel(const AttnParams p) 
     cp_commit();
   };
 
-  for (int m0 = 0; m0 < M_all; m0 += QR) {
-    // ---------------------------------------------------------------- one round of up to 64 query rows
+  {
+    // ---------------------------------------------------------------- this CTA's round of up to 64 query rows
+    const int m0 = blockIdx.z * QR;
     // query row m -> (head m / rows, block row m % rows); rows of this thread in row tile mt: lane/4 and +8
     int nv[2 * MT], gr[2 * MT], rr[2 * MT], hh[2 * MT];
     bool any_row = false;
@@ -147,9 +149,8 @@ __global__ void __launch_bounds__(THREADS) attn_span_kernel(const AttnParams p) 
       gr[i] = ok ? s_grp[rr[i]] : -1;
       any_row = any_row || nv[i] > span0;
     }
-    if (!__syncthreads_or(any_row)) continue;          // nobody in this round reaches the span
+    if (!__syncthreads_or(any_row)) return;            // nobody in this round reaches the span
 
-    __syncthreads();                                    // previous round done with every buffer
     for (int idx = threadIdx.x; idx < QR * CPR; idx += THREADS) {
       int row = idx / CPR, ch = idx % CPR, m = m0 + row;
       uint32_t off = S::OFF_Q + row * ROWB + ((ch ^ (row & 7)) << 4);
@@ -400,7 +401,8 @@ void launch_attention_tc(const ouro_model_desc &d, const void *q, const void *k_
   p.scale_log2 = 1.4426950408889634f / sqrtf((float)d.head_dim);
   p.part = part;
   p.out = (__nv_bfloat16 *)out;
-  dim3 grid((n_vis_max + SPAN - 1) / SPAN, d.n_kv_heads), mgrid(rows, (d.n_heads + 3) / 4);
+  const int m_all = (d.n_heads / d.n_kv_heads) * rows;      // query rows per kv head, served 64 per CTA
+  dim3 grid((n_vis_max + SPAN - 1) / SPAN, d.n_kv_heads, (m_all + QR - 1) / QR), mgrid(rows, (d.n_heads + 3) / 4);
   if (d.head_dim == 128) {
     launch_pdl(attn_span_kernel<128>, grid, THREADS, Smem<128>::BYTES, s, p);
     launch_pdl(attn_merge_kernel<128>, mgrid, 128, 0, s, p);
