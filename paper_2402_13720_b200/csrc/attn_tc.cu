@@ -150,6 +150,7 @@ __global__ void __launch_bounds__(THREADS) attn_span_kernel(const AttnParams p) 
       any_row = any_row || nv[i] > span0;
     }
     if (!__syncthreads_or(any_row)) return;            // nobody in this round reaches the span
+    const int n_mt = (min(QR, M_all - m0) + 15) >> 4;  // row tiles that hold query rows; the others are skipped
 
     for (int idx = threadIdx.x; idx < QR * CPR; idx += THREADS) {
       int row = idx / CPR, ch = idx % CPR, m = m0 + row;
@@ -221,6 +222,7 @@ __global__ void __launch_bounds__(THREADS) attn_span_kernel(const AttnParams p) 
           }
 #pragma unroll
           for (int mt = 0; mt < MT; ++mt) {
+            if (mt >= n_mt) continue;
             uint32_t a[4];
             int row = mt * 16 + (lane & 7) + ((mi & 1) << 3), ch = 2 * ks + (mi >> 1);
             ldsm_x4(sm_u + S::OFF_Q + row * ROWB + ((ch ^ (row & 7)) << 4), a[0], a[1], a[2], a[3]);
@@ -231,6 +233,7 @@ __global__ void __launch_bounds__(THREADS) attn_span_kernel(const AttnParams p) 
         // ---- mask by virtual position and group; warp-local row maxima (log2 domain)
 #pragma unroll
         for (int mt = 0; mt < MT; ++mt) {
+          if (mt >= n_mt) continue;
           const int iA = 2 * mt, iB = 2 * mt + 1;
           const int nA = (gid == -2 || gr[iA] == gid) ? nv[iA] : 0, nB = (gid == -2 || gr[iB] == gid) ? nv[iB] : 0;
           float mxA = -INFINITY, mxB = -INFINITY;
@@ -249,8 +252,8 @@ __global__ void __launch_bounds__(THREADS) attn_span_kernel(const AttnParams p) 
           mxB = fmaxf(mxB, __shfl_xor_sync(0xffffffffu, mxB, 1));
           mxB = fmaxf(mxB, __shfl_xor_sync(0xffffffffu, mxB, 2));
           if ((lane & 3) == 0) {
-            wmax[warp * QR + mt * 16 + (lane >> 2)] = mxA;
-            wmax[warp * QR + mt * 16 + (lane >> 2) + 8] = mxB;
+            wmax[(mt * 16 + (lane >> 2)) * WARPS + warp] = mxA;
+            wmax[(mt * 16 + (lane >> 2) + 8) * WARPS + warp] = mxB;
           }
         }
         __syncthreads();
@@ -258,12 +261,13 @@ __global__ void __launch_bounds__(THREADS) attn_span_kernel(const AttnParams p) 
         float scale_old[2 * MT];
 #pragma unroll
         for (int mt = 0; mt < MT; ++mt) {
+          if (mt >= n_mt) { scale_old[2 * mt] = scale_old[2 * mt + 1] = 1.f; continue; }
 #pragma unroll
           for (int hb = 0; hb < 2; ++hb) {
             const int i = 2 * mt + hb, row = mt * 16 + (lane >> 2) + 8 * hb;
-            float mc = wmax[row];
-#pragma unroll
-            for (int w = 1; w < WARPS; ++w) mc = fmaxf(mc, wmax[w * QR + row]);
+            const float4 m0v = *reinterpret_cast<const float4 *>(wmax + row * WARPS);
+            const float4 m1v = *reinterpret_cast<const float4 *>(wmax + row * WARPS + 4);
+            const float mc = fmaxf(fmaxf(fmaxf(m0v.x, m0v.y), fmaxf(m0v.z, m0v.w)), fmaxf(fmaxf(m1v.x, m1v.y), fmaxf(m1v.z, m1v.w)));
             const float mn = fmaxf(m_run[i], mc);
             scale_old[i] = (m_run[i] == -INFINITY) ? 0.f : exp2f(m_run[i] - mn);   // mn finite whenever m_run is
             m_run[i] = mn;
@@ -279,17 +283,18 @@ __global__ void __launch_bounds__(THREADS) attn_span_kernel(const AttnParams p) 
             }
             sum += __shfl_xor_sync(0xffffffffu, sum, 1);
             sum += __shfl_xor_sync(0xffffffffu, sum, 2);
-            if ((lane & 3) == 0) wsum[warp * QR + row] = sum;
+            if ((lane & 3) == 0) wsum[row * WARPS + warp] = sum;
           }
         }
         __syncthreads();
         // ---- running sums and O = O * scale + P V for this warp's slice of the head dimension
 #pragma unroll
         for (int i = 0; i < 2 * MT; ++i) {
+          if ((i >> 1) >= n_mt) continue;
           const int row = (i >> 1) * 16 + (lane >> 2) + 8 * (i & 1);
-          float add = wsum[row];
-#pragma unroll
-          for (int w = 1; w < WARPS; ++w) add += wsum[w * QR + row];
+          const float4 s0 = *reinterpret_cast<const float4 *>(wsum + row * WARPS);
+          const float4 s1 = *reinterpret_cast<const float4 *>(wsum + row * WARPS + 4);
+          const float add = ((((((s0.x + s0.y) + s0.z) + s0.w) + s1.x) + s1.y) + s1.z) + s1.w;    // warp order
           l_run[i] = l_run[i] * scale_old[i] + add;
         }
 #pragma unroll
@@ -312,6 +317,7 @@ __global__ void __launch_bounds__(THREADS) attn_span_kernel(const AttnParams p) 
           }
 #pragma unroll
           for (int mt = 0; mt < MT; ++mt) {
+            if (mt >= n_mt) continue;
             uint32_t a[4];
             int row = (lane & 7) + ((mi & 1) << 3), ch = 2 * kk + (mi >> 1);
             ldsm_x4(sm_u + S::OFF_P + (mt * 16 + row) * (CH * 2) + ((ch ^ (row & 7)) << 4), a[0], a[1], a[2], a[3]);
