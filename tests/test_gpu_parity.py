@@ -518,3 +518,37 @@ def test_verify_step_full_size_c2(L):
     pool.apply(ob.harvest_ops(tokens, o, P.gamma, P.S, P.K, A2, seq, len(acc2), P))
     assert gpu_pool_rows(eng) == pool_rows(pool)
     eng.close()
+
+
+# ------------------------------------------------------------ 7B-shaped pair: lossless at scale
+
+def test_c3_shapes_ouroboros_is_bit_identical_to_vanilla():
+    """Target 7B-shaped (32 layers), draft 1.1B-shaped (GQA 8:1, head_dim 64), bf16, replayed drafts and a
+    replayed phrase source: the generated text must equal plain greedy decoding on the same kernels bit for
+    bit, with phrase suffixes actually accepted along the way."""
+    T, D, P, R = synth.config("C3")
+    wt = synth.model_weights(T, 0, device="cuda:0")
+    wd = synth.model_weights(D, 100, device="cuda:0")
+    eng = binding.Engine(T, wt, P, D, wd)
+    prompt = synth.prompt(0, T.vocab, 96, R["copy_frac"], *R["span"])
+    gen = 72
+    van, _ = eng.generate_vanilla(prompt, gen)
+    truth = np.concatenate([prompt, van, np.zeros(64, dtype=np.int32)])
+
+    def drafter(seq, g, step):
+        d = synth.corrupt_drafts(5, truth, len(seq), g, T.vocab, 0.12, 0.03, step)
+        grams = np.empty((P.K, P.beta), dtype=np.int32)
+        for j in range(P.K):
+            grams[j, 0] = d[-1]
+            grams[j, 1:] = synth.corrupt_drafts(11 + j, truth, len(seq) + g, P.S, T.vocab, 0.08 * (j + 1), 0.0, step)
+        eng.phrase_update(grams[::-1])
+        return d
+
+    eng.set_drafter(drafter)
+    out, st = eng.generate(prompt, gen)
+    eng.set_drafter(None)
+    assert np.array_equal(out, van)
+    assert st["suffix_tokens"] > 0 and st["target_calls"] < gen // 2
+    nat, st2 = eng.generate(prompt, 24)                      # the draft model's own (chance-level) drafts
+    assert np.array_equal(nat, van[:24]) and st2["draft_calls"] == 4 * st2["target_calls"]
+    eng.close()
