@@ -301,12 +301,10 @@ extern "C" int ouro_assemble_candidates(ouro_ctx *c, const int32_t *draft_dev, c
   ModelRt &M = c->m[OURO_TARGET];
   const int gamma = c->p.gamma, S = c->p.beta - 1, K = c->p.K;
   if (M.L + 1 + gamma + K * S > M.d.max_seq) return fail(c, OURO_ECAPACITY, "cache length + block rows exceeds max_seq");
-  if (!suffix_dev) {
-    launch_pool_lookup(c->pool, draft_dev, gamma - 1, 0, K, c->cand_suffix, c->cand_count, c->stream);
-    suffix_dev = c->cand_suffix;
-    count_dev = c->cand_count;
-  }
-  launch_assemble_candidates(M.blk, c->st, draft_dev, suffix_dev, count_dev, M.L, gamma, S, K, c->stream);
+  if (!suffix_dev)
+    launch_lookup_assemble(c->pool, M.blk, c->st, draft_dev, c->cand_suffix, c->cand_count, M.L, gamma, S, K, c->stream);
+  else
+    launch_assemble_candidates(M.blk, c->st, draft_dev, suffix_dev, count_dev, M.L, gamma, S, K, c->stream);
   CKL();
   CK(cudaMemcpyAsync(c->pin, &c->st->n_rows, sizeof(int32_t), cudaMemcpyDeviceToHost, c->stream));
   CK(cudaStreamSynchronize(c->stream));
@@ -548,10 +546,8 @@ static int accept_step(ouro_ctx *c, const int32_t *argmax_dev, AcceptOut *r) {
     return fail(c, OURO_ESTATE, "no verified candidate block for the current cache length");
   const int gamma = c->p.gamma, S = c->p.beta - 1, L = T.L;
   cudaStream_t s = c->stream;
-  launch_accept(T.blk, c->st, argmax_dev, c->seq_dev, gamma, S, s);
-  launch_compact(T.d, T.k_cache, T.v_cache, c->st, L, gamma, S, s);
-  if (c->p.flags & (OURO_HARVEST_MATCHED | OURO_HARVEST_CANDIDATES | OURO_HARVEST_ACCEPTED))
-    launch_harvest(T.blk, c->st, c->pool, argmax_dev, c->seq_dev, gamma, S, c->p.flags, s);
+  launch_accept_compact_harvest(T.blk, c->st, c->pool, argmax_dev, c->seq_dev, T.d, T.k_cache, T.v_cache, L, gamma, S,
+                                c->p.flags, s);
   CKL();
   static_assert(sizeof(AcceptOut) <= PIN_INTS * 4, "pinned staging too small");
   CK(cudaMemcpyAsync(c->pin, &c->st->A, sizeof(AcceptOut), cudaMemcpyDeviceToHost, s));

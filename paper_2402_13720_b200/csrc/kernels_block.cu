@@ -155,8 +155,9 @@ void launch_pool_update(const PoolDev &P, DevState *st, const int32_t *ngrams, i
 // Eq. 7: rows [pending, d_1..d_gamma, p^1_2..beta, .., p^K'_2..beta].  Trunk row b: position L+b, sees
 // slots [0, L+b].  Suffix row (j, i): position L+gamma+i, sees slots [0, L+gamma] and its own
 // candidate's rows (j, 1..i), which sit at slots L+1+gamma+j*S .. (Eq. 8).
-__global__ void assemble_candidates_kernel(BlockDev b, DevState *st, const int32_t *draft, const int32_t *suffix,
-                                           const int32_t *count, int L, int gamma, int S, int K) {
+__device__ __forceinline__ void assemble_candidates_body(const BlockDev &b, DevState *st, const int32_t *draft,
+                                                         const int32_t *suffix, const int32_t *count, int L, int gamma,
+                                                         int S, int K) {
   int nc = S > 0 ? min(*count, K) : 0;
   int B = 1 + gamma + nc * S;
   int r = threadIdx.x;
@@ -189,6 +190,23 @@ __global__ void assemble_candidates_kernel(BlockDev b, DevState *st, const int32
   b.mask[2 * r + 1] = m1;
 }
 
+__global__ void assemble_candidates_kernel(BlockDev b, DevState *st, const int32_t *draft, const int32_t *suffix,
+                                           const int32_t *count, int L, int gamma, int S, int K) {
+  assemble_candidates_body(b, st, draft, suffix, count, L, gamma, S, K);
+}
+
+// Lookup with key d_gamma (warp 0) and packing in one launch.
+__global__ void lookup_assemble_kernel(PoolDev P, BlockDev b, DevState *st, const int32_t *draft, int32_t *suffix,
+                                       int32_t *count, int L, int gamma, int S, int K) {
+  if (threadIdx.x < 32) {
+    int32_t key = draft[gamma - 1];
+    int n = (key < 0 || P.S == 0) ? 0 : pool_lookup(P, key, K, suffix);
+    if (threadIdx.x == 0) *count = n;
+  }
+  __syncthreads();
+  assemble_candidates_body(b, st, draft, suffix, count, L, gamma, S, K);
+}
+
 __global__ void assemble_causal_kernel(BlockDev b, const int32_t *tokens, int n, int L) {
   int r = threadIdx.x;
   if (r >= n) return;
@@ -209,6 +227,11 @@ void launch_assemble_candidates(const BlockDev &b, DevState *st, const int32_t *
   OURO_COUNT_LAUNCH();
   assemble_candidates_kernel<<<1, OURO_MAX_ROWS, 0, s>>>(b, st, draft, suffix, count, L, gamma, S, K);
 }
+void launch_lookup_assemble(const PoolDev &P, const BlockDev &b, DevState *st, const int32_t *draft, int32_t *suffix,
+                            int32_t *count, int L, int gamma, int S, int K, cudaStream_t s) {
+  OURO_COUNT_LAUNCH();
+  lookup_assemble_kernel<<<1, OURO_MAX_ROWS, 0, s>>>(P, b, st, draft, suffix, count, L, gamma, S, K);
+}
 void launch_assemble_causal(const BlockDev &b, const int32_t *tokens, int n, int L, cudaStream_t s) {
   OURO_COUNT_LAUNCH();
   assemble_causal_kernel<<<1, OURO_MAX_ROWS, 0, s>>>(b, tokens, n, L);
@@ -219,8 +242,7 @@ void launch_assemble_causal(const BlockDev &b, const int32_t *tokens, int n, int
 // A == gamma): candidate j's chain is o[gamma], then the outputs at its own suffix rows; m_j counts
 // its leading suffix tokens equal to that chain; the largest m_j wins, earliest j on ties.  The step
 // accepts the matched tokens plus the chain's next output.  One thread: a few dozen comparisons.
-__global__ void accept_kernel(BlockDev b, DevState *st, const int32_t *o, int32_t *seq_dev, int gamma, int S) {
-  if (threadIdx.x != 0) return;
+__device__ void accept_body(const BlockDev &b, DevState *st, const int32_t *o, int32_t *seq_dev, int gamma, int S) {
   int nc = st->n_cand, A = 0, n = 0;
   while (A < gamma && b.tok[1 + A] == o[A]) ++A;
   for (int i = 0; i < A; ++i) st->accepted[n++] = b.tok[1 + i];
@@ -253,6 +275,10 @@ __global__ void accept_kernel(BlockDev b, DevState *st, const int32_t *o, int32_
   int base = st->n_seq;
   for (int i = 0; i < n; ++i) seq_dev[base + i] = st->accepted[i];
   st->n_seq = base + n;
+}
+
+__global__ void accept_kernel(BlockDev b, DevState *st, const int32_t *o, int32_t *seq_dev, int gamma, int S) {
+  if (threadIdx.x == 0) accept_body(b, st, o, seq_dev, gamma, S);
 }
 
 void launch_accept(const BlockDev &b, DevState *st, const int32_t *o, int32_t *seq_dev, int gamma, int S,
@@ -299,8 +325,8 @@ void launch_compact(const ouro_model_desc &d, void *k_cache, void *v_cache, cons
 //     following draft tokens agree with the target outputs for at least max(1, beta-2) positions, the
 //     beta-gram (t_s, o_s, .., o_{s+beta-2}) is inserted;
 //  3. extension: every beta-window of the text that ends inside the newly accepted tokens.
-__global__ void harvest_kernel(BlockDev b, DevState *st, PoolDev P, const int32_t *o, const int32_t *seq_dev,
-                               int gamma, int S, unsigned flags) {
+__device__ void harvest_body(const BlockDev &b, DevState *st, const PoolDev &P, const int32_t *o, const int32_t *seq_dev,
+                             int gamma, int S, unsigned flags) {
   const int beta = S + 1;
   int32_t ph[OURO_MAX_BETA], old[OURO_MAX_BETA];
   int A = st->A, nc = st->n_cand;
@@ -338,6 +364,58 @@ __global__ void harvest_kernel(BlockDev b, DevState *st, PoolDev P, const int32_
       pool_insert(P, st, ph);
     }
   }
+}
+
+__global__ void harvest_kernel(BlockDev b, DevState *st, PoolDev P, const int32_t *o, const int32_t *seq_dev,
+                               int gamma, int S, unsigned flags) {
+  harvest_body(b, st, P, o, seq_dev, gamma, S, flags);
+}
+
+// Acceptance, compaction and harvest in one launch.  Block 0: one thread accepts (Eq. 3, Eq. 9), then its first
+// warp harvests.  Blocks 1..: one (layer, K or V, suffix slot) each; every such block re-derives the chosen
+// candidate and its matched length from the block tokens and the outputs (a few dozen comparisons) instead of
+// waiting for block 0, then moves its cache row if the row belongs to the accepted suffix.
+__global__ void accept_compact_harvest_kernel(BlockDev b, DevState *st, PoolDev P, const int32_t *o, int32_t *seq_dev,
+                                              unsigned char *k_cache, unsigned char *v_cache, int L, int gamma, int S,
+                                              int max_seq, int row_bytes, unsigned flags) {
+  if (blockIdx.x == 0) {
+    if (threadIdx.x == 0) accept_body(b, st, o, seq_dev, gamma, S);
+    __syncthreads();
+    if (threadIdx.x < 32 && (flags & (OURO_HARVEST_MATCHED | OURO_HARVEST_CANDIDATES | OURO_HARVEST_ACCEPTED)))
+      harvest_body(b, st, P, o, seq_dev, gamma, S, flags);
+    return;
+  }
+  __shared__ int s_chosen, s_m;
+  if (threadIdx.x == 0) {
+    int nc = st->n_cand, A = 0, chosen = -1, best = -1;
+    while (A < gamma && b.tok[1 + A] == o[A]) ++A;
+    if (A == gamma)
+      for (int j = 0; j < nc; ++j) {
+        int base = 1 + gamma + j * S, mj = 0;
+        int32_t v = o[gamma];
+        while (mj < S && b.tok[base + mj] == v) { v = o[base + mj]; ++mj; }
+        if (mj > best) { best = mj; chosen = j; }
+      }
+    s_chosen = chosen;
+    s_m = best < 0 ? 0 : best;
+  }
+  __syncthreads();
+  const int idx = blockIdx.x - 1, t = idx % S, ly = idx / S;       // ly = 2 * layer + (0: K, 1: V)
+  if (s_chosen <= 0 || t >= s_m) return;                           // candidate 0 already sits next to the trunk
+  unsigned char *base = ((ly & 1) ? v_cache : k_cache) + (size_t)(ly >> 1) * max_seq * row_bytes;
+  const uint4 *src = (const uint4 *)(base + (size_t)(L + 1 + gamma + s_chosen * S + t) * row_bytes);
+  uint4 *dst = (uint4 *)(base + (size_t)(L + 1 + gamma + t) * row_bytes);
+  for (int i = threadIdx.x; i < row_bytes / 16; i += blockDim.x) dst[i] = src[i];
+}
+
+void launch_accept_compact_harvest(const BlockDev &b, DevState *st, const PoolDev &P, const int32_t *o, int32_t *seq_dev,
+                                   const ouro_model_desc &d, void *k_cache, void *v_cache, int L, int gamma, int S,
+                                   unsigned flags, cudaStream_t s) {
+  OURO_COUNT_LAUNCH();
+  const int es = d.dtype == OURO_BF16 ? 2 : 4;
+  accept_compact_harvest_kernel<<<1 + S * d.n_layers * 2, 128, 0, s>>>(b, st, P, o, seq_dev, (unsigned char *)k_cache,
+                                                                      (unsigned char *)v_cache, L, gamma, S, d.max_seq,
+                                                                      d.n_kv_heads * d.head_dim * es, flags);
 }
 
 void launch_harvest(const BlockDev &b, DevState *st, const PoolDev &P, const int32_t *o, const int32_t *seq_dev,

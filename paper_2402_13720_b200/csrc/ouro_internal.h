@@ -153,6 +153,11 @@ void launch_compact(const ouro_model_desc &d, void *k_cache, void *v_cache, cons
                     int S, cudaStream_t s);
 void launch_harvest(const BlockDev &b, DevState *st, const PoolDev &P, const int32_t *o, const int32_t *seq_dev,
                     int gamma, int S, unsigned flags, cudaStream_t s);
+void launch_lookup_assemble(const PoolDev &P, const BlockDev &b, DevState *st, const int32_t *draft, int32_t *suffix,
+                            int32_t *count, int L, int gamma, int S, int K, cudaStream_t s);
+void launch_accept_compact_harvest(const BlockDev &b, DevState *st, const PoolDev &P, const int32_t *o, int32_t *seq_dev,
+                                   const ouro_model_desc &d, void *k_cache, void *v_cache, int L, int gamma, int S,
+                                   unsigned flags, cudaStream_t s);
 void launch_argmax(const float *logits, int rows, int vocab, int32_t *out, cudaStream_t s);
 void launch_pick_token(const int32_t *src, int index, int32_t *dst, cudaStream_t s);
 void launch_set_state(DevState *st, int32_t *seq_dev, int n_seq, int pending, int fill, cudaStream_t s);
