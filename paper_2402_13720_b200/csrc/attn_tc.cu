@@ -71,6 +71,23 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   return *reinterpret_cast<uint32_t *>(&t);
 }
 
+// Dense query-row index m -> (block row, query head inside the kv group).  Groups are contiguous row ranges;
+// group G with rows [a, b) owns the indices [g*a, g*b), ordered head-major inside the group.
+__device__ __forceinline__ void map_row(int m, int g, int rows, const int *grp, int &row, int &hq) {
+  int a = 0;
+  while (true) {
+    int b = a + 1;
+    while (b < rows && grp[b] == grp[a]) ++b;
+    if (m < g * b || b >= rows) {
+      int e = m - g * a, n = b - a;
+      hq = e / n;
+      row = a + e % n;
+      return;
+    }
+    a = b;
+  }
+}
+
 template <int HD>
 struct Smem {
   static constexpr int ROWB = HD * 2;                              // bytes per K/V/Q tile row
@@ -82,7 +99,8 @@ struct Smem {
   static constexpr int OFF_WSUM = OFF_WMAX + WARPS * QR * 4;
   static constexpr int OFF_NVIS = OFF_WSUM + WARPS * QR * 4;       // [OURO_MAX_ROWS]
   static constexpr int OFF_GRP = OFF_NVIS + OURO_MAX_ROWS * 4;
-  static constexpr int BYTES = OFF_GRP + OURO_MAX_ROWS * 4;
+  static constexpr int OFF_MAP = OFF_GRP + OURO_MAX_ROWS * 4;      // [QR] block row | head << 16 of each query row
+  static constexpr int BYTES = OFF_MAP + QR * 4;
 };
 
 template <int HD>
@@ -95,7 +113,7 @@ __global__ void __launch_bounds__(THREADS) attn_span_kernel(const AttnParams p) 
   constexpr int NT2 = DW / 8;                  // 8-dim MMA tiles per warp
   extern __shared__ __align__(128) uint8_t smem[];
   float *wmax = (float *)(smem + S::OFF_WMAX), *wsum = (float *)(smem + S::OFF_WSUM);
-  int *s_nvis = (int *)(smem + S::OFF_NVIS), *s_grp = (int *)(smem + S::OFF_GRP);
+  int *s_nvis = (int *)(smem + S::OFF_NVIS), *s_grp = (int *)(smem + S::OFF_GRP), *s_map = (int *)(smem + S::OFF_MAP);
   const uint32_t sm_u = smem_u32(smem);
 
   pdl_trigger();
@@ -136,17 +154,27 @@ __global__ void __launch_bounds__(THREADS) attn_span_kernel(const AttnParams p) 
   {
     // ---------------------------------------------------------------- this CTA's round of up to 64 query rows
     const int m0 = blockIdx.z * QR;
-    // query row m -> (head m / rows, block row m % rows); rows of this thread in row tile mt: lane/4 and +8
+    // Query rows are ordered group by group (a group's rows for head 0, then for head 1, ..), so that the 64 rows
+    // of a round belong to few groups and the chunk that holds block keys needs few passes.  Rows of this thread
+    // in row tile mt: lane/4 and +8.
+    if (threadIdx.x < QR) {
+      int r0 = 0, hq = 0;
+      if (m0 + (int)threadIdx.x < M_all) map_row(m0 + threadIdx.x, g, p.rows, s_grp, r0, hq);
+      s_map[threadIdx.x] = r0 | (hq << 16);
+    }
+    __syncthreads();
     int nv[2 * MT], gr[2 * MT], rr[2 * MT], hh[2 * MT];
     bool any_row = false;
 #pragma unroll
     for (int i = 0; i < 2 * MT; ++i) {
-      int m = m0 + (i >> 1) * 16 + (lane >> 2) + (i & 1) * 8;
-      bool ok = m < M_all;
-      rr[i] = ok ? m % p.rows : 0;
-      hh[i] = kvh * g + (ok ? m / p.rows : 0);
-      nv[i] = ok ? s_nvis[rr[i]] : 0;
-      gr[i] = ok ? s_grp[rr[i]] : -1;
+      int ml = (i >> 1) * 16 + (lane >> 2) + (i & 1) * 8;
+      rr[i] = 0; hh[i] = kvh * g; nv[i] = 0; gr[i] = -1;
+      if (m0 + ml < M_all) {
+        rr[i] = s_map[ml] & 0xffff;
+        hh[i] = kvh * g + (s_map[ml] >> 16);
+        nv[i] = s_nvis[rr[i]];
+        gr[i] = s_grp[rr[i]];
+      }
       any_row = any_row || nv[i] > span0;
     }
     if (!__syncthreads_or(any_row)) return;            // nobody in this round reaches the span
@@ -156,7 +184,7 @@ __global__ void __launch_bounds__(THREADS) attn_span_kernel(const AttnParams p) 
       int row = idx / CPR, ch = idx % CPR, m = m0 + row;
       uint32_t off = S::OFF_Q + row * ROWB + ((ch ^ (row & 7)) << 4);
       if (m < M_all)
-        cp_async16(sm_u + off, p.q + (size_t)(m % p.rows) * p.H * HD + (kvh * g + m / p.rows) * HD + ch * 8);
+        cp_async16(sm_u + off, p.q + (size_t)(s_map[row] & 0xffff) * p.H * HD + (kvh * g + (s_map[row] >> 16)) * HD + ch * 8);
       else
         *reinterpret_cast<uint4 *>(smem + off) = make_uint4(0, 0, 0, 0);
     }
@@ -205,6 +233,11 @@ __global__ void __launch_bounds__(THREADS) attn_span_kernel(const AttnParams p) 
           cp_wait_all();
           __syncthreads();
         }
+        // row tiles none of whose rows takes part in this pass are left alone (same decision in every warp)
+        bool live[MT];
+#pragma unroll
+        for (int mt = 0; mt < MT; ++mt)
+          live[mt] = mt < n_mt && (gid == -2 || __ballot_sync(0xffffffffu, gr[2 * mt] == gid || gr[2 * mt + 1] == gid) != 0);
         // ---- S = Q K^T for this warp's 16 keys, all row tiles
         float s[MT][2][4];
 #pragma unroll
@@ -222,7 +255,7 @@ __global__ void __launch_bounds__(THREADS) attn_span_kernel(const AttnParams p) 
           }
 #pragma unroll
           for (int mt = 0; mt < MT; ++mt) {
-            if (mt >= n_mt) continue;
+            if (!live[mt]) continue;
             uint32_t a[4];
             int row = mt * 16 + (lane & 7) + ((mi & 1) << 3), ch = 2 * ks + (mi >> 1);
             ldsm_x4(sm_u + S::OFF_Q + row * ROWB + ((ch ^ (row & 7)) << 4), a[0], a[1], a[2], a[3]);
@@ -233,7 +266,7 @@ __global__ void __launch_bounds__(THREADS) attn_span_kernel(const AttnParams p) 
         // ---- mask by virtual position and group; warp-local row maxima (log2 domain)
 #pragma unroll
         for (int mt = 0; mt < MT; ++mt) {
-          if (mt >= n_mt) continue;
+          if (!live[mt]) continue;
           const int iA = 2 * mt, iB = 2 * mt + 1;
           const int nA = (gid == -2 || gr[iA] == gid) ? nv[iA] : 0, nB = (gid == -2 || gr[iB] == gid) ? nv[iB] : 0;
           float mxA = -INFINITY, mxB = -INFINITY;
@@ -261,7 +294,7 @@ __global__ void __launch_bounds__(THREADS) attn_span_kernel(const AttnParams p) 
         float scale_old[2 * MT];
 #pragma unroll
         for (int mt = 0; mt < MT; ++mt) {
-          if (mt >= n_mt) { scale_old[2 * mt] = scale_old[2 * mt + 1] = 1.f; continue; }
+          if (!live[mt]) { scale_old[2 * mt] = scale_old[2 * mt + 1] = 1.f; continue; }
 #pragma unroll
           for (int hb = 0; hb < 2; ++hb) {
             const int i = 2 * mt + hb, row = mt * 16 + (lane >> 2) + 8 * hb;
@@ -290,7 +323,7 @@ __global__ void __launch_bounds__(THREADS) attn_span_kernel(const AttnParams p) 
         // ---- running sums and O = O * scale + P V for this warp's slice of the head dimension
 #pragma unroll
         for (int i = 0; i < 2 * MT; ++i) {
-          if ((i >> 1) >= n_mt) continue;
+          if (!live[i >> 1]) continue;
           const int row = (i >> 1) * 16 + (lane >> 2) + 8 * (i & 1);
           const float4 s0 = *reinterpret_cast<const float4 *>(wsum + row * WARPS);
           const float4 s1 = *reinterpret_cast<const float4 *>(wsum + row * WARPS + 4);
@@ -317,7 +350,7 @@ __global__ void __launch_bounds__(THREADS) attn_span_kernel(const AttnParams p) 
           }
 #pragma unroll
           for (int mt = 0; mt < MT; ++mt) {
-            if (mt >= n_mt) continue;
+            if (!live[mt]) continue;
             uint32_t a[4];
             int row = (lane & 7) + ((mi & 1) << 3), ch = 2 * kk + (mi >> 1);
             ldsm_x4(sm_u + S::OFF_P + (mt * 16 + row) * (CH * 2) + ((ch ^ (row & 7)) << 4), a[0], a[1], a[2], a[3]);
@@ -389,6 +422,22 @@ int attention_tc_setup() {
   if (cudaFuncSetAttribute(attn_span_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, Smem<64>::BYTES) != cudaSuccess)
     return OURO_ECUDA;
   return OURO_OK;
+}
+
+// Folds the per-span pieces written by either span kernel (head dim 64 or 128) into the block's attention output.
+void launch_attention_merge(const ouro_model_desc &d, const BlockDev &b, int rows, float *part, void *out, cudaStream_t s) {
+  OURO_COUNT_LAUNCH();
+  AttnParams p{};
+  p.lin_end = b.lin_end; p.seg_start = b.seg_start; p.seg_len = b.seg_len; p.group = b.group;
+  p.rows = rows; p.H = d.n_heads; p.Hkv = d.n_kv_heads;
+  p.cap = (d.max_seq + SPAN - 1) / SPAN;
+  p.part = part;
+  p.out = (__nv_bfloat16 *)out;
+  dim3 mgrid(rows, (d.n_heads + 3) / 4);
+  if (d.head_dim == 128)
+    launch_pdl(attn_merge_kernel<128>, mgrid, 128, 0, s, p);
+  else
+    launch_pdl(attn_merge_kernel<64>, mgrid, 128, 0, s, p);
 }
 
 // n_vis_max: an upper bound of the number of keys any row of the block sees (cache length + rows).

@@ -738,6 +738,8 @@ struct FastModel {
   bool ok = false;
   std::vector<LayerMaps> layers;
   CUtensorMap head;
+  CUtensorMap kmap, vmap;               // K and V caches as [layers * max_seq][kv width], box 64 x 128 (tcgen05 attention)
+  bool kv_maps = false;
   CUtensorMap x_d[8], x_q[8], x_f[8];   // activations normed [128, d], attention out [128, dq], SwiGLU out [128, F]; box rows 16, 32, .., 128
 };
 struct FastState {
@@ -812,7 +814,7 @@ int ouro_fast_setup(ouro_ctx *c) {
   f->s.attn_part = (float *)((char *)f->s.ss + ss_bytes());
   if (cudaMemsetAsync(f->s.counters, 0, 2 * MAX_TILES * sizeof(int), c->stream) != cudaSuccess ||
       cudaFuncSetAttribute(gemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess ||
-      attention_tc_setup() != OURO_OK) {
+      attention_tc_setup() != OURO_OK || attention_tm_setup() != OURO_OK) {
     delete f;
     c->err = "tensor-core GEMM set-up failed";
     return OURO_ECUDA;
@@ -833,6 +835,10 @@ int ouro_fast_setup(ouro_ctx *c) {
            make_map(&lm.wd, M.w_down[l], d.d_model, d.d_ffn, TILE_N);
     }
     ok = ok && make_map(&fm.head, M.lm_head, d.vocab, d.d_model, TILE_N);
+    if (ok && attention_tm_supported(d)) {
+      ok = make_map(&fm.kmap, M.k_cache, d.n_layers * d.max_seq, dkv, 128) && make_map(&fm.vmap, M.v_cache, d.n_layers * d.max_seq, dkv, 128);
+      fm.kv_maps = ok;
+    }
     for (int i = 0; i < 8 && ok; ++i)
       ok = make_map(&fm.x_d[i], c->a.xn, OURO_MAX_ROWS, d.d_model, 16 * (i + 1)) &&
            make_map(&fm.x_q[i], c->a.att, OURO_MAX_ROWS, dq, 16 * (i + 1)) &&
@@ -956,7 +962,11 @@ int ouro_fast_layer(ouro_ctx *c, int which, int l, int rows) {
   }
   {
     ProfScope ps(c, OURO_PROF_ATTENTION);
-    if (attention_tc_supported(d))
+    if (c->fast->s.m[which].kv_maps) {
+      launch_attention_tm(d, a.q, &c->fast->s.m[which].kmap, &c->fast->s.m[which].vmap, M.k_cache, M.v_cache, M.blk, rows, M.L,
+                          M.L + rows, l, c->fast->s.attn_part, &c->st->status, s);
+      launch_attention_merge(d, M.blk, rows, c->fast->s.attn_part, a.att, s);
+    } else if (attention_tc_supported(d))
       launch_attention_tc(d, a.q, M.k_cache, M.v_cache, M.blk, rows, M.L, M.L + rows, l, c->fast->s.attn_part, a.att, s);
     else
       launch_attention_simple(d, a.q, M.k_cache, M.v_cache, M.blk, rows, l, a.att, s);
