@@ -75,6 +75,7 @@ struct TmParams {
   const __nv_bfloat16 *k, *v;      // this layer's cache: [max_seq][Hkv*HD]
   const int32_t *lin_end, *seg_start, *seg_len, *group;
   int rows, H, Hkv, L, cap, row0;  // row0: first row of this layer in the tensor maps
+  int n_spans;
   float scale_log2;
   float *part;                     // [rows][H][cap][HD+2]: max (log2 domain), sum, unnormalised output
   int *status;
@@ -175,8 +176,9 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tm_kernel(const __grid_consta
   const uint32_t sm_u = smem_u32(smem);
   Misc *ms = reinterpret_cast<Misc *>(smem + OFF_MISC);
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  // the last span goes first: it holds the block's own keys and takes one pass per group
-  const int sc = gridDim.x - 1 - blockIdx.x, kvh = blockIdx.y, m0 = blockIdx.z * QR;
+  // blockIdx.x walks (span, kv head) with the last span of every head first: it holds the block's own keys and
+  // takes one pass per group, so it should not be what the grid ends on
+  const int sc = p.n_spans - 1 - blockIdx.x / p.Hkv, kvh = blockIdx.x % p.Hkv, m0 = blockIdx.y * QR;
   const int g = p.H / p.Hkv, dkv = p.Hkv * HD, M_all = g * p.rows, span0 = sc * SPAN;
 
   if (sm_u & 1023) {                                   // the swizzled tiles need a 1024-byte aligned base
@@ -583,6 +585,7 @@ void launch_attention_tm(const ouro_model_desc &d, const void *q, const void *km
   p.part = part;
   p.status = status;
   const int m_all = (d.n_heads / d.n_kv_heads) * rows;
-  dim3 grid((n_vis_max + SPAN - 1) / SPAN, d.n_kv_heads, (m_all + QR - 1) / QR);
+  p.n_spans = (n_vis_max + SPAN - 1) / SPAN;
+  dim3 grid(p.n_spans * d.n_kv_heads, (m_all + QR - 1) / QR);
   launch_pdl(attn_tm_kernel, grid, THREADS, SMEM_BYTES, s, p);
 }
