@@ -238,6 +238,7 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_tc_kernel(const __grid_consta
   volatile int *abort_flag = (volatile int *)(bars + 37);
   volatile int *wait_flag = (volatile int *)(bars + 39);   // [2]: outcome of the epilogue's accumulator wait
   float *rs = (float *)(bars + 48);                         // [128] per-token factor 1/rms of the consumed activations
+  int *spos = (int *)(rs + OURO_MAX_ROWS);                  // [128] token positions (rotary table rows), QKV epilogue
 
   pdl_trigger();
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -454,51 +455,107 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_tc_kernel(const __grid_consta
                   acc[j].x += tmp[cc][j].x; acc[j].y += tmp[cc][j].y; acc[j].z += tmp[cc][j].z; acc[j].w += tmp[cc][j].w;
                 }
             }
+            // What the epilogue reads (residual stream, rotary table) is fetched for the four tokens at once,
+            // ahead of the arithmetic and the stores: one round trip to L2 per pass instead of one per token.
+            const bool full4 = 4 * ng + 3 < valid;
+            if (p.mode == MODE_RESIDUAL && p.gain) {
+              float4 yv[4];
+#pragma unroll
+              for (int j = 0; j < 4; ++j) {
+                const int t = tb + j * n * 4;
+                yv[j] = make_float4(0.f, 0.f, 0.f, 0.f);
+                if (t < p.rows) {
+                  const float *y = p.out_f32 + (size_t)t * p.ldo + col;
+                  if (full4) {
+                    yv[j] = *reinterpret_cast<const float4 *>(y);
+                  } else {
+                    if (4 * ng < valid) yv[j].x = y[0];
+                    if (4 * ng + 1 < valid) yv[j].y = y[1];
+                    if (4 * ng + 2 < valid) yv[j].z = y[2];
+                  }
+                }
+              }
+              float gn[4];
+#pragma unroll
+              for (int e = 0; e < 4; ++e) gn[e] = 4 * ng + e < valid ? __bfloat162float(p.gain[col + e]) : 0.f;
+#pragma unroll
+              for (int j = 0; j < 4; ++j) {
+                const int t = tb + j * n * 4;
+                if (t >= p.rows) continue;                            // uniform inside the warp
+                float *y = p.out_f32 + (size_t)t * p.ldo + col;
+                const float yn[4] = {yv[j].x + acc[j].x, yv[j].y + acc[j].y, yv[j].z + acc[j].z, yv[j].w + acc[j].w};
+                float sq = 0.f;
+#pragma unroll
+                for (int e = 0; e < 4; ++e)
+                  if (4 * ng + e < valid) sq += yn[e] * yn[e];
+                if (full4) {
+                  *reinterpret_cast<float4 *>(y) = make_float4(yn[0], yn[1], yn[2], yn[3]);
+                  __nv_bfloat162 lo = __floats2bfloat162_rn(gn[0] * yn[0], gn[1] * yn[1]);
+                  __nv_bfloat162 hi = __floats2bfloat162_rn(gn[2] * yn[2], gn[3] * yn[3]);
+                  *reinterpret_cast<uint2 *>(p.xb + (size_t)t * p.ldo + col) = make_uint2(*(uint32_t *)&lo, *(uint32_t *)&hi);
+                } else {
+#pragma unroll
+                  for (int e = 0; e < 4; ++e)
+                    if (4 * ng + e < valid) {
+                      y[e] = yn[e];
+                      p.xb[(size_t)t * p.ldo + col + e] = __float2bfloat16_rn(gn[e] * yn[e]);
+                    }
+                }
+#pragma unroll
+                for (int o = 16; o; o >>= 1) sq += __shfl_xor_sync(0xffffffffu, sq, o);
+                if (lane == 0) p.ss_out[(size_t)tile * OURO_MAX_ROWS + t] = sq;
+              }
+              continue;
+            }
+            if (p.mode == MODE_QKV) {
+              const int cm = row0 + 4 * ng;                      // first of this thread's 4 columns inside q, k or v
+              const int half = p.head_dim >> 1;
+              const bool upper = (cm & half) != 0;
+              float4 cs4[4], sn4[4];
+#pragma unroll
+              for (int j = 0; j < 4; ++j) {
+                const int t = tb + j * n * 4;
+                cs4[j] = sn4[j] = make_float4(0.f, 0.f, 0.f, 0.f);
+                if (t < p.rows && seg != 2) {
+                  const size_t ti = (size_t)spos[t] * half + (cm & (half - 1));
+                  cs4[j] = *reinterpret_cast<const float4 *>(p.cos_t + ti);
+                  sn4[j] = *reinterpret_cast<const float4 *>(p.sin_t + ti);
+                }
+              }
+#pragma unroll
+              for (int j = 0; j < 4; ++j) {
+                const int t = tb + j * n * 4;
+                if (t >= p.rows) continue;                            // uniform inside the warp
+                const float r = rs[t];
+                const float vals[4] = {acc[j].x * r, acc[j].y * r, acc[j].z * r, acc[j].w * r};
+                float other[4];
+#pragma unroll
+                for (int e = 0; e < 4; ++e) other[e] = __shfl_xor_sync(0xffffffffu, vals[e], half >> 2);
+                const float cs[4] = {cs4[j].x, cs4[j].y, cs4[j].z, cs4[j].w}, sn[4] = {sn4[j].x, sn4[j].y, sn4[j].z, sn4[j].w};
+                float rv[4];
+#pragma unroll
+                for (int e = 0; e < 4; ++e)
+                  rv[e] = seg == 2 ? vals[e] : (upper ? vals[e] * cs[e] + other[e] * sn[e] : vals[e] * cs[e] - other[e] * sn[e]);
+                __nv_bfloat16 *dst = seg == 0 ? p.q_out + (size_t)t * p.dq + cm
+                                   : seg == 1 ? p.k_out + (size_t)(p.L + t) * p.dkv + cm
+                                              : p.v_out + (size_t)(p.L + t) * p.dkv + cm;
+                if (full4) {
+                  __nv_bfloat162 lo = __floats2bfloat162_rn(rv[0], rv[1]), hi = __floats2bfloat162_rn(rv[2], rv[3]);
+                  *reinterpret_cast<uint2 *>(dst) = make_uint2(*(uint32_t *)&lo, *(uint32_t *)&hi);
+                } else {
+#pragma unroll
+                  for (int e = 0; e < 4; ++e)
+                    if (4 * ng + e < valid) dst[e] = __float2bfloat16_rn(rv[e]);
+                }
+              }
+              continue;
+            }
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
               const int t = tb + j * n * 4;
               if (t >= p.rows) continue;                              // uniform inside the warp
-              if (p.mode == MODE_RESIDUAL && p.gain) {
-                float *y = p.out_f32 + (size_t)t * p.ldo + col;
-                const float add[4] = {acc[j].x, acc[j].y, acc[j].z, acc[j].w};
-                float sq = 0.f;
-#pragma unroll
-                for (int e = 0; e < 4; ++e)
-                  if (4 * ng + e < valid) {
-                    const float yn = y[e] + add[e];
-                    y[e] = yn;
-                    p.xb[(size_t)t * p.ldo + col + e] = __float2bfloat16_rn(__bfloat162float(p.gain[col + e]) * yn);
-                    sq += yn * yn;
-                  }
-#pragma unroll
-                for (int o = 16; o; o >>= 1) sq += __shfl_xor_sync(0xffffffffu, sq, o);
-                if (lane == 0) p.ss_out[(size_t)tile * OURO_MAX_ROWS + t] = sq;
-                continue;
-              }
               const float r = rs[t];
               const float vals[4] = {acc[j].x * r, acc[j].y * r, acc[j].z * r, acc[j].w * r};
-              if (p.mode == MODE_QKV) {
-                const int cm = row0 + 4 * ng;                    // first of this thread's 4 columns inside q, k or v
-                const int half = p.head_dim >> 1;
-                float other[4];
-#pragma unroll
-                for (int e = 0; e < 4; ++e) other[e] = __shfl_xor_sync(0xffffffffu, vals[e], half >> 2);
-                const bool upper = (cm & half) != 0;
-                const size_t ti = (size_t)p.pos[t] * half + (cm & (half - 1));
-#pragma unroll
-                for (int e = 0; e < 4; ++e) {
-                  if (4 * ng + e >= valid) continue;
-                  if (seg == 2) {
-                    p.v_out[(size_t)(p.L + t) * p.dkv + cm + e] = __float2bfloat16_rn(vals[e]);
-                  } else {
-                    const float cs = p.cos_t[ti + e], sn = p.sin_t[ti + e];
-                    const float rv = upper ? vals[e] * cs + other[e] * sn : vals[e] * cs - other[e] * sn;
-                    if (seg == 0) p.q_out[(size_t)t * p.dq + cm + e] = __float2bfloat16_rn(rv);
-                    else p.k_out[(size_t)(p.L + t) * p.dkv + cm + e] = __float2bfloat16_rn(rv);
-                  }
-                }
-                continue;
-              }
               if (p.mode == MODE_HEAD) {                              // the warp's 32 lanes hold the tile's 128 columns
                 uint32_t bu = 0;
                 int bi = col;
@@ -541,6 +598,7 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_tc_kernel(const __grid_consta
         r = 1.0f / sqrtf(sum * p.ss_inv_d + p.eps);
       }
       rs[et] = r;
+      spos[et] = (p.mode == MODE_QKV && et < p.rows) ? p.pos[et] : 0;
     }
     epi_barrier();
 
@@ -631,7 +689,7 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_tc_kernel(const __grid_consta
                     const int t = t0 + i;
                     if (t < p.rows) {
                       const float other = xchg[i * TILE_N + (nl ^ half)];
-                      const size_t ti = (size_t)p.pos[t] * half + ih;
+                      const size_t ti = (size_t)spos[t] * half + ih;
                       const float cs = p.cos_t[ti], sn = p.sin_t[ti];
                       const float r = upper ? v[i] * cs + other * sn : v[i] * cs - other * sn;
                       if (seg == 0) p.q_out[(size_t)t * p.dq + cm] = __float2bfloat16_rn(r);
@@ -762,7 +820,7 @@ size_t ss_bytes() { return (size_t)MAX_SS_TILES * OURO_MAX_ROWS * sizeof(float);
 
 int stages_for(int t_pad, int smem_max) {
   int stage = A_BYTES + t_pad * BLOCK_K * 2;
-  int fixed = 1024 + 64 * OURO_MAX_ROWS * 4 + 1024;  // alignment slack, exchange buffer, barriers, flags, per-token factors
+  int fixed = 1024 + 64 * OURO_MAX_ROWS * 4 + 1536;  // alignment slack, exchange buffer, barriers, flags, per-token factors and positions
   int s = (smem_max - fixed) / stage;
   return s > 12 ? 12 : s;
 }
