@@ -25,6 +25,14 @@ import numpy as np
 import torch
 
 ROOT = os.path.dirname(os.path.abspath(__file__))
+GEMM_TRAFFIC_BYTES = 138.3e6          # dram read + write per gemm_tc_kernel launch, mean of the step's five launches (ncu)
+GEMM_TRAFFIC_REV = "69d5e3358c94bdac"  # sha256 prefix of csrc/gemm_tc.cu the counters were taken on
+
+
+def kernel_rev():
+    import hashlib
+    with open(os.path.join(ROOT, "paper_2402_13720_b200", "csrc", "gemm_tc.cu"), "rb") as f:
+        return hashlib.sha256(f.read()).hexdigest()[:16]
 if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
@@ -385,9 +393,13 @@ def main():
     gemm_bytes = sum(wl.bytes["per_class"][c] * prof[c][1] for c in gemm)
     achieved = gemm_bytes / (gemm_ms * 1e-3) / 1e9 if gemm_ms > 0 else 0.0
     fwd_ms = prof["forward"][0]
+    # DRAM bytes per launch (read + write) of the five GEMM launches from one ncu capture of this workload
+    # (profiles/gemm_tc_kernel_verify_step_c2.md); it belongs to GEMM_TRAFFIC_REV of the kernel source and
+    # is reported as null once the kernel has changed since.
+    traffic = GEMM_TRAFFIC_BYTES if kernel_rev() == GEMM_TRAFFIC_REV and args.cache_len == 4096 else None
     roofline = {"bound": "hbm", "kernel": "gemm_tc_kernel", "launches_per_step": gemm_launches,
                 "achieved": achieved, "peak": peak, "peak_kind": peak_kind, "unit": "GB/s",
-                "frac": achieved / peak, "traffic": None,
+                "frac": achieved / peak, "traffic": traffic,
                 "bytes_per_launch": gemm_bytes / max(1, gemm_launches), "us_per_launch": gemm_ms * 1e3 / max(1, gemm_launches),
                 "kernel_us": {c: round(prof[c][0] * 1e3, 2) for c in PROF_CLASSES},
                 "forward_us": round(fwd_ms * 1e3, 2),
