@@ -19,8 +19,9 @@
 //
 // A chunk that holds the block's own keys is processed once per group (trunk, each candidate), each pass with a
 // tile of its own: cache slots equal virtual positions for the prefix and the trunk, so the tile the TMA fetched
-// is already right for them; for a candidate, warp 0 copies its suffix rows over the tile before the pass.  Rows
-// of other groups sit the pass out.
+// is already right for them; for a candidate, warp 0 copies its suffix rows over the tile before the pass (the
+// tile is fetched once per stage; what an earlier candidate left in rows beyond a pass's own keys is masked).
+// Rows of other groups sit the pass out.
 // The value computed for a query depends only on (virtual position -> key) and on the fixed chunk and span
 // boundaries, never on the other rows of the block: a token gets bit-identical attention whether it is verified
 // inside a candidate block or decoded alone.
@@ -67,7 +68,7 @@ constexpr int SMEM_BYTES = OFF_MISC + 3072;
 static_assert(sizeof(Misc) <= 3072, "misc area");
 
 // work item: chunk | group ordinal (63: every row) << 3 | flags
-enum { IT_PATCH = 1 << 9 };
+enum { IT_PATCH = 1 << 9, IT_REUSE = 1 << 10 };   // REUSE: the stage already holds this chunk's tile
 
 struct TmParams {
   CUtensorMap kmap, vmap;          // [layers * max_seq][Hkv * HD] bf16, box 64 x 128, 128-byte swizzle
@@ -266,11 +267,14 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tm_kernel(const __grid_consta
         if (c0 + CH <= p.L) {
           ms->items[n++] = ci | (63 << 3);
         } else {
+          // the chunk's tile is fetched into both stages once; later passes only patch their rows over it
+          int in_chunk = 0;
           for (int o = 0; o < ng; ++o) {
             if (ms->gmax[o] <= c0) continue;
             const int last = ms->gs[o + 1] - 1, len = ms->len[last], lin = ms->lin[last];
             const bool patch = len > 0 && lin < c0 + CH && lin + len > c0;
-            ms->items[n++] = ci | (o << 3) | (patch ? IT_PATCH : 0);
+            ms->items[n++] = ci | (o << 3) | (patch ? IT_PATCH : 0) | (in_chunk >= 2 ? IT_REUSE : 0);
+            ++in_chunk;
           }
         }
       }
@@ -323,7 +327,10 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tm_kernel(const __grid_consta
         const int it = ms->items[i], ci = it & 7, go = (it >> 3) & 63, st = i & 1;
         if (i >= early) {
           if (i >= 2) ok = mbar_wait(&ms->empty[st], ((i >> 1) - 1) & 1, ms, p.status) && ok;
-          if (lane == 0) request_tile(i, ci);
+          if (lane == 0) {
+            if (it & IT_REUSE) mbar_arrive(&ms->full[st]);   // nothing to fetch: the phase completes at once
+            else request_tile(i, ci);
+          }
         }
         if (it & IT_PATCH) {
           // a candidate's pass: its suffix rows go over the tile the TMA fetched (slots = positions up to the trunk)
