@@ -471,25 +471,28 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tm_kernel(const __grid_consta
         ok = mbar_wait(&ms->s_ready[b], (i >> 1) & 1, ms, p.status) && ok;
         fence_after_sync();
         float alpha = 1.f;
-        const int nk = active ? nv - c0 : 0;           // keys of this chunk the row sees: tile columns below nk
+        const int nk = active ? min(nv - c0, CH) : 0;  // keys of this chunk the row sees: tile columns below nk
+        const int nk_w = __reduce_max_sync(0xffffffffu, nk);
         const bool whole = __all_sync(0xffffffffu, !active || nk >= CH);   // no score of an active row is masked
-        if (__any_sync(0xffffffffu, active)) {         // TMEM loads are warp-wide: every lane takes part
+        if (nk_w > 0) {                                // TMEM loads are warp-wide: every lane takes part
+          // a half of the chunk that no row of the warp reaches takes no arithmetic (its scores are read all the same)
+          const bool need_own = h * 64 < nk_w;
           // ---- row maximum over the chunk (scaling by a positive factor commutes with max, bit for bit)
           float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
           for (int hh = 0; hh < 2; ++hh) {
-            float v[64];
-            tmem_ld32_issue(lane_addr + b * 128 + hh * 64, v);
-            tmem_ld32_issue(lane_addr + b * 128 + hh * 64 + 32, v + 32);
-            tmem_ld_wait32(v);
-            tmem_ld_wait32(v + 32);
+            float vm[64];
+            tmem_ld32_issue(lane_addr + b * 128 + hh * 64, vm);
+            tmem_ld32_issue(lane_addr + b * 128 + hh * 64 + 32, vm + 32);
+            tmem_ld_wait32(vm);
+            tmem_ld_wait32(vm + 32);
             if (whole) {
 #pragma unroll
-              for (int j = 0; j < 64; ++j) mx4[j & 3] = fmaxf(mx4[j & 3], v[j]);
-            } else {
+              for (int j = 0; j < 64; ++j) mx4[j & 3] = fmaxf(mx4[j & 3], vm[j]);
+            } else if (hh * 64 < nk_w) {
 #pragma unroll
               for (int j = 0; j < 64; ++j)
-                if (hh * 64 + j < nk) mx4[j & 3] = fmaxf(mx4[j & 3], v[j]);
+                if (hh * 64 + j < nk) mx4[j & 3] = fmaxf(mx4[j & 3], vm[j]);
             }
           }
           const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
@@ -500,7 +503,9 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tm_kernel(const __grid_consta
           tmem_ld32_issue(lane_addr + b * 128 + h * 64 + 32, v + 32);
           tmem_ld_wait32(v);
           tmem_ld_wait32(v + 32);
-          if (active) {
+          float sum = 0.f;
+          uint8_t *prow = smem + OFF_P + b * TILE + h * HALF + t * 128;   // this thread's 128 bytes of P
+          if (active && need_own) {
             float sum4[4] = {0.f, 0.f, 0.f, 0.f};      // four interleaved partial sums, folded in a fixed order
             uint32_t w[32];
             if (whole) {
@@ -521,11 +526,15 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tm_kernel(const __grid_consta
                 w[j >> 1] = pack_bf16(p0, p1);
               }
             }
-            const float sum = (sum4[0] + sum4[1]) + (sum4[2] + sum4[3]);
+            sum = (sum4[0] + sum4[1]) + (sum4[2] + sum4[3]);
 #pragma unroll
             for (int q8 = 0; q8 < 8; ++q8)              // 16-byte piece q8 of key half h: keys 64 h + 8 q8 ..
-              *reinterpret_cast<uint4 *>(smem + OFF_P + b * TILE + h * HALF + t * 128 + ((q8 ^ (t & 7)) << 4)) =
-                  make_uint4(w[4 * q8], w[4 * q8 + 1], w[4 * q8 + 2], w[4 * q8 + 3]);
+              *reinterpret_cast<uint4 *>(prow + ((q8 ^ (t & 7)) << 4)) = make_uint4(w[4 * q8], w[4 * q8 + 1], w[4 * q8 + 2], w[4 * q8 + 3]);
+          } else if (active) {
+#pragma unroll
+            for (int q8 = 0; q8 < 8; ++q8) *reinterpret_cast<uint4 *>(prow + (q8 << 4)) = make_uint4(0u, 0u, 0u, 0u);
+          }
+          if (active) {
             alpha = (m_run == -INFINITY) ? 0.f : ex2(m_run - mn);
             l_run = l_run * alpha + sum;
             m_run = mn;
