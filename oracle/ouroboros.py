@@ -15,6 +15,8 @@ What the paper fixes and what is this build's reading:
   * Ties for "the phrase with the largest accepted suffix" go to the earliest candidate.
   * The phrase pool's layout, capacity, eviction and ordering are not given by the paper: a
     sets x ways table addressed by the first token, LRU by a global stamp (PhrasePool below).
+  * Phrase-level drafting on the draft model (Section 3.1) is not specified by the paper; PhraseDrafter
+    is this build's reading: the draft model verifies pool phrases on itself, Section 3.2 style.
   * "Sub-segments of the discarded draft that match the verification" (Section 3.3) is read as
     in harvest_ops(); the replacement of tried phrases by their verified versions follows the
     second paragraph of Section 3.3.
@@ -273,6 +275,61 @@ class ModelDrafter:
             c.length = L + n
             feed = [int(tf.argmax_rows(logits[-1:])[0])]
             out.append(feed[0])
+        return out
+
+    def rollback(self, valid_len):
+        self.cache.length = min(self.cache.length, valid_len)
+
+
+def draft_accept(tokens, o, n, S, n_cand):
+    """One phrase-level drafting round of the draft model.  Rows 0..n-1 of the block are text the draft
+    model is being fed (nothing to verify there), so its next greedy token is o[n-1]; candidate j's
+    chain continues from it exactly as in Eq. 9.  Returns (j_star, m, gained): the chosen candidate
+    (-1 without candidates), its matched suffix tokens, and the 1 + m tokens the round yields."""
+    if n_cand == 0:
+        return -1, 0, [int(o[n - 1])]
+    best = (-1, -1, None)
+    for j in range(n_cand):
+        base, m, v = n + j * S, 0, o[n - 1]
+        while m < S and tokens[base + m] == v:
+            v = o[base + m]
+            m += 1
+        if m > best[1]:
+            best = (j, m, v)
+    j, m, v = best
+    return j, m, [int(t) for t in tokens[n + j * S:n + j * S + m]] + [int(v)]
+
+
+class PhraseDrafter:
+    """Phrase-level drafting on the draft model (Section 3.1, Eq. 6: gamma draft tokens for gamma / c
+    draft forwards).  The paper gives no procedure ("we will not go into detail ..."), so this is this
+    build's reading: a drafting round is the verification step of Section 3.2 run by the DRAFT model on
+    itself.  The round's block is the text the draft model has not cached yet followed by the K pool
+    phrases that start with the last known token, under the mask of Eq. 8; the draft model's greedy
+    outputs accept the longest matching phrase prefix (Eq. 9) plus one more token.  The drafts are, by
+    Eq. 4 applied to the draft model, the ones token-level drafting (Eq. 1) would produce; only the
+    number of draft forwards changes.  The pool is read, never written, while drafting."""
+
+    def __init__(self, W, P, pool):
+        self.W, self.P, self.pool, self.cache = W, P, pool, tf.KVCache(W.desc)
+        self.calls = 0
+
+    def draft(self, seq, gamma, step):
+        c, S, out = self.cache, self.P.S, []
+        feed = [int(t) for t in seq[c.length:]]
+        while len(out) < gamma:
+            n, L = len(feed), c.length
+            cands = self.pool.lookup(feed[-1], self.P.K) if S > 0 else []
+            tokens, pos, group, visible = build_block(L, feed[0], feed[1:], cands)
+            o = tf.argmax_rows(tf.forward(self.W, c, tokens, pos, visible))
+            self.calls += 1
+            j, m, gained = draft_accept(tokens, o, n, S, len(cands))
+            keep = min(len(gained), gamma - len(out))       # a draft has exactly gamma tokens
+            mk = min(m, keep)                                # kept tokens whose K/V the round computed
+            compact(c, L, n - 1, S, n - 1, j, mk)
+            c.length = L + n + mk
+            out += gained[:keep]
+            feed = [out[-1]]
         return out
 
     def rollback(self, valid_len):

@@ -302,3 +302,86 @@ def test_eos_stops_generation(c1):
     P = dataclasses.replace(C1P, eos_token=eos)
     out, _ = ob.generate(W, ob.ModelDrafter(Wd), prompt, 30, P)
     assert out == cut == ob.vanilla_greedy(W, prompt, 30, eos=eos)
+
+
+# ------------------------------------------------------------------- phrase-level drafting (Section 3.1)
+
+class _Spy:
+    """Runs two drafters side by side on the same calls and records what each returned."""
+
+    def __init__(self, a, b):
+        self.a, self.b, self.log = a, b, []
+
+    def draft(self, seq, gamma, step):
+        da, db = self.a.draft(seq, gamma, step), self.b.draft(seq, gamma, step)
+        self.log.append((da, db))
+        return da
+
+    def rollback(self, valid_len):
+        self.a.rollback(valid_len)
+        self.b.rollback(valid_len)
+
+
+@pytest.mark.parametrize("seed", [0, 3])
+def test_phrase_drafter_gives_the_token_level_drafts(c1, seed):
+    """Eq. 4 applied to the draft model: drafting by phrases changes how many forwards the draft model runs,
+    never what it drafts.  The token-level drafter (Eq. 1) is the independent definition."""
+    W, Wd = c1
+    prompt = synth.prompt(seed, C1T.vocab, C1R["n"], C1R["copy_frac"], *C1R["span"])
+    pool = ob.PhrasePool(C1P.pool_sets, C1P.pool_ways, C1P.beta)
+    tok, phr = ob.ModelDrafter(Wd), ob.PhraseDrafter(Wd, C1P, pool)
+    spy = _Spy(tok, phr)
+    out, stats = ob.generate(W, spy, prompt, 40, C1P, pool=pool)
+    assert out == ob.vanilla_greedy(W, prompt, 40)
+    assert all(a == b and len(b) == C1P.gamma for a, b in spy.log)
+    assert phr.calls <= C1P.gamma * stats["target_calls"]
+    assert tok.cache.length >= phr.cache.length - 1           # the phrase drafter may also hold d_gamma
+
+
+def test_phrase_drafter_saves_forwards_when_the_pool_knows_the_continuation(c1):
+    """A pool phrase equal to the draft model's own greedy continuation is accepted whole: one forward yields
+    1 + S tokens (c of Eq. 6 above 1); a pool of wrong phrases costs nothing but yields one token per forward."""
+    W, Wd = c1
+    P = C1P
+    prompt = [int(t) for t in synth.prompt(5, C1T.vocab, 20, 0.0, 4, 4)]
+    cont = ob.vanilla_greedy(Wd, prompt, P.gamma + 2)          # the draft model's own greedy text
+    good = ob.PhrasePool(P.pool_sets, P.pool_ways, P.beta)
+    good.insert([prompt[-1]] + cont[:P.S])
+    d = ob.PhraseDrafter(Wd, P, good)
+    assert d.draft(prompt, P.gamma, 0) == cont[:P.gamma]
+    assert d.calls == -(-P.gamma // (P.S + 1))                # ceil(gamma / (1 + S)) rounds
+    bad = ob.PhrasePool(P.pool_sets, P.pool_ways, P.beta)
+    bad.insert([prompt[-1]] + [(cont[0] + 1) % C1T.vocab] * P.S)
+    d2 = ob.PhraseDrafter(Wd, P, bad)
+    assert d2.draft(prompt, P.gamma, 0) == cont[:P.gamma] and d2.calls == P.gamma
+
+
+def test_phrase_drafter_cache_equals_fresh_prefill(c1):
+    """After rounds that accepted phrase suffixes the draft cache holds exactly the K/V of its text."""
+    W, Wd = c1
+    P = C1P
+    prompt = [int(t) for t in synth.prompt(6, C1T.vocab, 20, 0.0, 4, 4)]
+    cont = ob.vanilla_greedy(Wd, prompt, 8)
+    pool = ob.PhrasePool(P.pool_sets, P.pool_ways, P.beta)
+    pool.insert([prompt[-1]] + [(cont[0] + 1) % C1T.vocab] * P.S)      # tried first (newest last -> insert order below)
+    pool.insert([prompt[-1]] + cont[:P.S])
+    pool.insert([prompt[-1]] + [(cont[0] + 2) % C1T.vocab] * P.S)      # newest: candidate 0, wrong; the good one is candidate 1
+    d = ob.PhraseDrafter(Wd, P, pool)
+    out = d.draft(prompt, P.gamma, 0)
+    assert out == cont[:P.gamma]
+    text = prompt + out
+    n = d.cache.length
+    fresh = tf.KVCache(C1D)
+    tf.forward(Wd, fresh, text[:n], list(range(n)), tf.causal_visible(0, n))
+    assert n >= len(prompt) + P.S and np.abs(d.cache.k[:, :n] - fresh.k[:, :n]).max() < 1e-12
+    assert np.abs(d.cache.v[:, :n] - fresh.v[:, :n]).max() < 1e-12
+
+
+def test_draft_accept_planted_mistake():
+    """Chain of Eq. 9 on the draft side: the first suffix token is checked against o[n-1], not against o[n]."""
+    S, n = 3, 2
+    tokens = [7, 8, 20, 21, 22, 20, 30, 31]                  # trunk 7 8; candidates (20 21 22), (20 30 31)
+    o = [0, 20, 21, 99, 0, 30, 31, 55]                       # after 8 comes 20; cand 0 matches 2, cand 1 matches 3
+    assert ob.draft_accept(tokens, o, n, S, 2) == (1, 3, [20, 30, 31, 55])
+    assert ob.draft_accept(tokens, o, n, S, 1) == (0, 2, [20, 21, 99])
+    assert ob.draft_accept(tokens, o, n, S, 0) == (-1, 0, [20])
