@@ -50,7 +50,8 @@ enum {
   OURO_HARVEST_MATCHED = 1,     /* Section 3.3, first part: matched sub-segments of the discarded draft */
   OURO_HARVEST_CANDIDATES = 2,  /* Section 3.3, second part: tried phrases replaced by their verified version */
   OURO_HARVEST_ACCEPTED = 4,    /* extension: beta-grams ending inside the newly accepted tokens */
-  OURO_SEED_PROMPT = 8          /* extension: beta-grams of the prompt enter the pool at prefill */
+  OURO_SEED_PROMPT = 8,         /* extension: beta-grams of the prompt enter the pool at prefill */
+  OURO_DRAFT_PHRASES = 16       /* Section 3.1: the draft model drafts phrase by phrase (see ouro_draft) */
 };
 
 typedef struct ouro_ctx ouro_ctx;
@@ -179,7 +180,14 @@ int ouro_accept_and_compact(ouro_ctx *ctx, const int32_t *argmax_dev, int32_t *n
 /* Advances model `which` past the first n rows of its current causal block (they become cached text). */
 int ouro_advance(ouro_ctx *ctx, int which, int32_t n);
 
-/* Eq. 1: gamma greedy draft tokens from the draft model (or the external drafter) into draft_dev [gamma]. */
+/* Eq. 1: gamma greedy draft tokens from the draft model (or the external drafter) into draft_dev [gamma].
+ * With OURO_DRAFT_PHRASES (and no external drafter) the draft model drafts phrase by phrase (Section 3.1,
+ * Eq. 6).  The paper does not give the procedure; here a drafting round is the verification step of Section
+ * 3.2 run by the draft model on itself: the text it has not cached yet, followed by the K pool phrases that
+ * start with the last known token, go through one draft forward under the mask of Eq. 8; the draft model's
+ * greedy outputs accept the longest matching phrase prefix (Eq. 9) and one more token, and its cache is
+ * compacted like the target's.  The tokens are those of token-level drafting; only the number of draft
+ * forwards (ouro_stats.draft_calls) changes.  The pool is read, not written, while drafting. */
 int ouro_draft(ouro_ctx *ctx, int32_t *draft_dev);
 
 /* Whole loops.  out_host [max_new]; *n_out tokens written (stops at eos_token).  ouro_generate is the

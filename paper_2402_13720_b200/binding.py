@@ -23,7 +23,7 @@ OURO_OK, OURO_EINVAL, OURO_ENOMEM, OURO_ECAPACITY, OURO_ECUDA, OURO_ETIMEOUT, OU
 OURO_F32, OURO_BF16 = 0, 1
 OURO_TARGET, OURO_DRAFT = 0, 1
 OURO_MAX_ROWS, OURO_MAX_BETA, OURO_MAX_K, OURO_MAX_GAMMA = 128, 16, 16, 32
-OURO_HARVEST_MATCHED, OURO_HARVEST_CANDIDATES, OURO_HARVEST_ACCEPTED, OURO_SEED_PROMPT = 1, 2, 4, 8
+OURO_HARVEST_MATCHED, OURO_HARVEST_CANDIDATES, OURO_HARVEST_ACCEPTED, OURO_SEED_PROMPT, OURO_DRAFT_PHRASES = 1, 2, 4, 8, 16
 
 
 class ModelDescC(C.Structure):
@@ -128,7 +128,8 @@ def desc_c(m: synth.ModelDesc) -> ModelDescC:
 
 def params_c(p: synth.DecodeParams) -> ParamsC:
     flags = (OURO_HARVEST_MATCHED if p.harvest_matched else 0) | (OURO_HARVEST_CANDIDATES if p.harvest_candidates else 0) | \
-            (OURO_HARVEST_ACCEPTED if p.harvest_accepted else 0) | (OURO_SEED_PROMPT if p.seed_prompt else 0)
+            (OURO_HARVEST_ACCEPTED if p.harvest_accepted else 0) | (OURO_SEED_PROMPT if p.seed_prompt else 0) | \
+            (OURO_DRAFT_PHRASES if getattr(p, "draft_phrases", False) else 0)
     return ParamsC(p.gamma, p.beta, p.K, p.pool_sets, p.pool_ways, flags, p.eos_token)
 
 

@@ -581,6 +581,47 @@ extern "C" int ouro_accept_and_compact(ouro_ctx *c, const int32_t *argmax_dev, i
 // which yields d_1; each further token costs one single-row forward.  With an external drafter the
 // tokens come from the callback; a present draft model still runs the same forwards on them, so that
 // replayed drafts cost what real drafting costs.
+// Section 3.1 (see ouro_draft in the header): the draft model drafts phrase by phrase.  Every round is one draft
+// forward over the text it has not cached yet plus the pool phrases that start with the last known token, and
+// yields one token plus the matched phrase prefix.  Two small reads per round tell the host the block's row
+// count and how far the draft and its cache advanced.
+static int draft_step_phrases(ouro_ctx *c, int32_t *out_dev, int *calls) {
+  const int gamma = c->p.gamma, S = c->p.beta - 1, K = c->p.K;
+  ModelRt &D = c->m[OURO_DRAFT];
+  cudaStream_t s = c->stream;
+  const int n_seq = (int)c->seq.size();
+  if (n_seq + gamma + K * S > D.d.max_seq) return fail(c, OURO_ECAPACITY, "draft cache full");
+  // text that does not fit the first round's block beside the candidates goes through plain causal blocks
+  if (n_seq - D.L + K * S > OURO_MAX_ROWS) TRY(feed_text(c, OURO_DRAFT, n_seq - 1, nullptr));
+  int have = 0;
+  while (have < gamma) {
+    const int n = have == 0 ? n_seq - D.L : 1;
+    const int32_t *tokens = have == 0 ? c->seq_dev + D.L : out_dev + have - 1;
+    if (n < 1) return fail(c, OURO_ESTATE, "draft cache ahead of the text");
+    launch_draft_lookup_assemble(c->pool, D.blk, c->st, tokens, n, c->cand_suffix, c->cand_count, D.L, S, K, s);
+    CKL();
+    CK(cudaMemcpyAsync(c->pin, &c->st->n_rows, sizeof(int32_t), cudaMemcpyDeviceToHost, s));
+    CK(cudaStreamSynchronize(s));
+    D.blk_rows = c->pin[0];
+    D.blk_L = D.L;
+    D.blk_is_candidate = true;
+    if (D.blk_rows < n || D.blk_rows > n + K * S) return fail(c, OURO_ECUDA, "draft block has an impossible row count");
+    TRY(forward(c, OURO_DRAFT, c->a.argmax, nullptr));
+    launch_draft_accept_compact(D.blk, c->st, c->a.argmax, out_dev, have, gamma, D.d, D.k_cache, D.v_cache, D.L, n, S, s);
+    CKL();
+    CK(cudaMemcpyAsync(c->pin, &c->st->d_keep, 2 * sizeof(int32_t), cudaMemcpyDeviceToHost, s));
+    CK(cudaStreamSynchronize(s));
+    const int keep = c->pin[0], cached = c->pin[1];
+    if (keep < 1 || keep > gamma - have || cached < 0 || cached > keep)
+      return fail(c, OURO_ECUDA, "drafting round returned an impossible count");
+    D.L += n + cached;
+    D.blk_rows = 0;
+    have += keep;
+    *calls += 1;
+  }
+  return OURO_OK;
+}
+
 static int draft_step(ouro_ctx *c, int32_t *out_dev, int *calls) {
   const int gamma = c->p.gamma;
   ModelRt &D = c->m[OURO_DRAFT];
@@ -597,6 +638,7 @@ static int draft_step(ouro_ctx *c, int32_t *out_dev, int *calls) {
     CK(cudaStreamSynchronize(c->stream));   // the pinned staging is reused by later calls
   }
   if (!D.present) return OURO_OK;
+  if (!ext && (c->p.flags & OURO_DRAFT_PHRASES)) return draft_step_phrases(c, out_dev, calls);
   if ((int)c->seq.size() + gamma > D.d.max_seq) return fail(c, OURO_ECAPACITY, "draft cache full");
   int last = 0;
   TRY(feed_text(c, OURO_DRAFT, (int)c->seq.size(), &last));

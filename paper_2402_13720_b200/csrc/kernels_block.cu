@@ -418,6 +418,104 @@ void launch_accept_compact_harvest(const BlockDev &b, DevState *st, const PoolDe
                                                                       d.n_kv_heads * d.head_dim * es, flags);
 }
 
+// ------------------------------------------------------------- phrase-level drafting (Section 3.1)
+// A drafting round of the draft model.  Rows 0..n-1 are text it is fed (tokens[0..n-1], no verification needed),
+// then the suffixes of up to K pool phrases that start with tokens[n-1], packed as in Eq. 7 / Eq. 8 with the
+// n text rows in the role of the trunk.
+__global__ void draft_lookup_assemble_kernel(PoolDev P, BlockDev b, DevState *st, const int32_t *tokens, int n,
+                                             int32_t *suffix, int32_t *count, int L, int S, int K) {
+  if (threadIdx.x < 32) {
+    int32_t key = tokens[n - 1];
+    int found = (key < 0 || P.S == 0 || S == 0) ? 0 : pool_lookup(P, key, K, suffix);
+    if (threadIdx.x == 0) *count = found;
+  }
+  __syncthreads();
+  const int nc = S > 0 ? min(*count, K) : 0, B = n + nc * S, r = threadIdx.x;
+  if (r == 0) {
+    st->n_cand = nc;
+    st->n_rows = B;
+  }
+  if (r >= B) return;
+  u64 m0 = 0, m1 = 0;
+  if (r < n) {
+    b.tok[r] = tokens[r];
+    b.pos[r] = L + r;
+    b.group[r] = 0;
+    b.lin_end[r] = L + r + 1;
+    b.seg_start[r] = 0;
+    b.seg_len[r] = 0;
+    for (int c = 0; c <= r; ++c) (c < 64 ? m0 : m1) |= 1ull << (c & 63);
+  } else {
+    const int j = (r - n) / S, i = (r - n) % S + 1;
+    b.tok[r] = suffix[j * S + i - 1];
+    b.pos[r] = L + n - 1 + i;
+    b.group[r] = 1 + j;
+    b.lin_end[r] = L + n;
+    b.seg_start[r] = L + n + j * S;
+    b.seg_len[r] = i;
+    for (int c = 0; c < n; ++c) (c < 64 ? m0 : m1) |= 1ull << (c & 63);
+    for (int c = n + j * S; c <= r; ++c) (c < 64 ? m0 : m1) |= 1ull << (c & 63);
+  }
+  b.mask[2 * r] = m0;
+  b.mask[2 * r + 1] = m1;
+}
+
+// The round's outcome.  The draft model's next greedy token is o[n-1]; candidate j's chain continues from it as
+// in Eq. 9; the longest match wins (earliest on ties) and the round yields its m tokens plus the chain's next
+// one, cut to what the draft still lacks.  Block 0 writes the tokens; blocks 1.. each re-derive the choice and
+// move one row of the draft cache next to the text (candidate 0 already sits there).
+__global__ void draft_accept_compact_kernel(BlockDev b, DevState *st, const int32_t *o, int32_t *out_dev, int have,
+                                            int gamma, unsigned char *k_cache, unsigned char *v_cache, int L, int n, int S,
+                                            int max_seq, int row_bytes) {
+  __shared__ int s_chosen, s_m;
+  __shared__ int32_t s_bonus;
+  if (threadIdx.x == 0) {
+    const int nc = st->n_cand;
+    int chosen = -1, best = -1;
+    int32_t bonus = o[n - 1];
+    for (int j = 0; j < nc; ++j) {
+      int base = n + j * S, mj = 0;
+      int32_t v = o[n - 1];
+      while (mj < S && b.tok[base + mj] == v) { v = o[base + mj]; ++mj; }
+      if (mj > best) { best = mj; chosen = j; bonus = v; }
+    }
+    s_chosen = chosen;
+    s_m = best < 0 ? 0 : best;
+    s_bonus = bonus;
+  }
+  __syncthreads();
+  const int m = s_m, keep = min(m + 1, gamma - have), cached = min(m, keep);
+  if (blockIdx.x == 0) {
+    if (threadIdx.x < keep) out_dev[have + threadIdx.x] = (int)threadIdx.x < m ? b.tok[n + s_chosen * S + threadIdx.x] : s_bonus;
+    if (threadIdx.x == 0) {
+      st->d_keep = keep;
+      st->d_cached = cached;
+    }
+    return;
+  }
+  const int idx = blockIdx.x - 1, t = idx % S, ly = idx / S;       // ly = 2 * layer + (0: K, 1: V)
+  if (s_chosen <= 0 || t >= cached) return;
+  unsigned char *base = ((ly & 1) ? v_cache : k_cache) + (size_t)(ly >> 1) * max_seq * row_bytes;
+  const uint4 *src = (const uint4 *)(base + (size_t)(L + n + s_chosen * S + t) * row_bytes);
+  uint4 *dst = (uint4 *)(base + (size_t)(L + n + t) * row_bytes);
+  for (int i = threadIdx.x; i < row_bytes / 16; i += blockDim.x) dst[i] = src[i];
+}
+
+void launch_draft_lookup_assemble(const PoolDev &P, const BlockDev &b, DevState *st, const int32_t *tokens, int n,
+                                  int32_t *suffix, int32_t *count, int L, int S, int K, cudaStream_t s) {
+  OURO_COUNT_LAUNCH();
+  draft_lookup_assemble_kernel<<<1, OURO_MAX_ROWS, 0, s>>>(P, b, st, tokens, n, suffix, count, L, S, K);
+}
+void launch_draft_accept_compact(const BlockDev &b, DevState *st, const int32_t *o, int32_t *out_dev, int have, int gamma,
+                                 const ouro_model_desc &d, void *k_cache, void *v_cache, int L, int n, int S,
+                                 cudaStream_t s) {
+  OURO_COUNT_LAUNCH();
+  const int es = d.dtype == OURO_BF16 ? 2 : 4;
+  draft_accept_compact_kernel<<<1 + (S > 0 ? S : 0) * d.n_layers * 2, 128, 0, s>>>(
+      b, st, o, out_dev, have, gamma, (unsigned char *)k_cache, (unsigned char *)v_cache, L, n, S, d.max_seq,
+      d.n_kv_heads * d.head_dim * es);
+}
+
 void launch_harvest(const BlockDev &b, DevState *st, const PoolDev &P, const int32_t *o, const int32_t *seq_dev,
                     int gamma, int S, unsigned flags, cudaStream_t s) {
   OURO_COUNT_LAUNCH();

@@ -53,6 +53,9 @@ struct DevState {
   int32_t status;    // sticky device-side error word (0 = fine)
   int32_t pad;
   u64 clock;         // phrase-pool stamp counter
+  // last phrase-level drafting round of the draft model (Section 3.1)
+  int32_t d_keep;    // draft tokens the round added (at most what was still missing of gamma)
+  int32_t d_cached;  // how many of them have their K/V in the draft cache (matched suffix tokens kept)
 };
 
 // Per-row description of a query block.  Row r attends, in this order, cache slots [0, lin_end[r])
@@ -158,6 +161,11 @@ void launch_lookup_assemble(const PoolDev &P, const BlockDev &b, DevState *st, c
 void launch_accept_compact_harvest(const BlockDev &b, DevState *st, const PoolDev &P, const int32_t *o, int32_t *seq_dev,
                                    const ouro_model_desc &d, void *k_cache, void *v_cache, int L, int gamma, int S,
                                    unsigned flags, cudaStream_t s);
+void launch_draft_lookup_assemble(const PoolDev &P, const BlockDev &b, DevState *st, const int32_t *tokens, int n,
+                                  int32_t *suffix, int32_t *count, int L, int S, int K, cudaStream_t s);
+void launch_draft_accept_compact(const BlockDev &b, DevState *st, const int32_t *o, int32_t *out_dev, int have, int gamma,
+                                 const ouro_model_desc &d, void *k_cache, void *v_cache, int L, int n, int S,
+                                 cudaStream_t s);
 void launch_argmax(const float *logits, int rows, int vocab, int32_t *out, cudaStream_t s);
 void launch_pick_token(const int32_t *src, int index, int32_t *dst, cudaStream_t s);
 void launch_set_state(DevState *st, int32_t *seq_dev, int n_seq, int pending, int fill, cudaStream_t s);

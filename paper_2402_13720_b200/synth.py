@@ -125,6 +125,7 @@ class DecodeParams:
     harvest_candidates: bool = True   # corrected candidates (Section 3.3, second paragraph)
     harvest_accepted: bool = True     # beta-grams of the accepted text (extension, off in paper-pure mode)
     seed_prompt: bool = True          # beta-grams of the prompt (extension, off in paper-pure mode)
+    draft_phrases: bool = False       # the draft model drafts phrase by phrase (Section 3.1)
     eos_token: int = -1
 
     @property

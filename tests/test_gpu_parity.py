@@ -552,3 +552,58 @@ def test_c3_shapes_ouroboros_is_bit_identical_to_vanilla():
     nat, st2 = eng.generate(prompt, 24)                      # the draft model's own (chance-level) drafts
     assert np.array_equal(nat, van[:24]) and st2["draft_calls"] == 4 * st2["target_calls"]
     eng.close()
+
+
+# ------------------------------------------------------------------- phrase-level drafting (Section 3.1)
+
+def test_phrase_level_drafting_c1_matches_oracle():
+    """The draft model drafts phrase by phrase: same text, same target calls and the oracle's number of draft
+    forwards; against token-level drafting on the GPU only the number of draft forwards may differ."""
+    import dataclasses
+    P = dataclasses.replace(C1P, draft_phrases=True)
+    w = synth.model_weights(C1T, 0, device="cuda:0")
+    eng = binding.Engine(C1T, w, P, C1D, w)
+    tok = binding.Engine(C1T, w, C1P, C1D, w)
+    W = tf.Weights(C1T, synth.model_weights(C1T, 0))
+    Wd = tf.Weights(C1D, synth.model_weights(C1T, 0))
+    fewer = 0
+    for seed in (0, 1, 4):
+        prompt = synth.prompt(seed, C1T.vocab, C1R["n"], C1R["copy_frac"], *C1R["span"])
+        gen = C1R["gen"]
+        out, stats = eng.generate(prompt, gen)
+        pool_gpu = gpu_pool_rows(eng)
+        pool = oracle_pool(P)
+        drafter = ob.PhraseDrafter(Wd, P, pool)
+        trace = []
+        ref, rstats = ob.generate(W, drafter, prompt, gen, P, pool=pool, trace=trace)
+        assert out.tolist() == ref
+        assert stats["target_calls"] == rstats["target_calls"] and stats["draft_calls"] == drafter.calls
+        assert stats["suffix_tokens"] == sum(rstats["m"]) and stats["candidates"] == sum(rstats["n_cand"])
+        assert pool_gpu[0] == [list(p) for _, p in trace[-1]["pool"]]
+        out2, stats2 = tok.generate(prompt, gen)
+        assert np.array_equal(out, out2) and stats2["target_calls"] == stats["target_calls"]
+        assert stats2["draft_calls"] == P.gamma * stats2["target_calls"] >= stats["draft_calls"]
+        fewer += stats2["draft_calls"] - stats["draft_calls"]
+    assert fewer > 0                                   # some round did accept a phrase on the draft side
+    eng.close()
+    tok.close()
+
+
+def test_phrase_level_drafting_bf16_self_draft():
+    """bf16 on the tensor-core path, the target's own weights as the draft model: drafts are always accepted, the
+    pool fills with the text's own phrases, and drafting by phrases must leave text and target calls untouched."""
+    import dataclasses
+    P0 = synth.DecodeParams(4, 9, 4, 32, 8)
+    P1 = dataclasses.replace(P0, draft_phrases=True)
+    w = synth.model_weights(MIDB, 3, device="cuda:0")
+    prompt = synth.prompt(3, MIDB.vocab, 96, 0.3, 8, 32)
+    res = []
+    for P in (P0, P1):
+        eng = binding.Engine(MIDB, w, P, MIDB, w)
+        van, _ = eng.generate_vanilla(prompt, 120)
+        out, st = eng.generate(prompt, 120)
+        assert np.array_equal(out, van)
+        res.append(st)
+        eng.close()
+    assert res[0]["target_calls"] == res[1]["target_calls"] and res[0]["full_accepts"] == res[0]["target_calls"]
+    assert res[1]["draft_calls"] <= res[0]["draft_calls"] == 4 * res[0]["target_calls"]
