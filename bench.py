@@ -297,6 +297,17 @@ def run_generate(args, device):
     e = 2 if T.dtype == "bf16" else 4
     wbytes = T.n_layers * T.layer_weight_elems() * e + T.vocab * T.d_model * e
     peaks = {}
+    # Phrase-level drafting on the draft model (Section 3.1): same weights and caches of their own, the draft model's
+    # own drafts.  What changes is the number of draft forwards per target call (gamma / c of Eq. 6); with
+    # random-init models c stays near 1 unless the draft model's text repeats.
+    eng2 = binding.Engine(T, wt, dataclasses.replace(P, draft_phrases=True), D, wd, device=device)
+    out, st = eng2.generate(prompt, gen)
+    res["natural_phrase_drafting"] = {
+        "tokens_per_s": len(out) / (st["ms_total"] * 1e-3), "target_calls": st["target_calls"], "draft_calls": st["draft_calls"],
+        "draft_forwards_per_target_call": st["draft_calls"] / st["target_calls"],
+        "ms_draft_per_step": st["ms_draft"] / st["target_calls"], "identical_to_vanilla": bool(np.array_equal(out, van))}
+    eng2.close()
+
     try:
         peaks = json.load(open(os.path.join(ROOT, "MEASURED_PEAKS.json")))
     except Exception:

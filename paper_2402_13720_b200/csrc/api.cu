@@ -1,6 +1,8 @@
 // C ABI of libouro: context set-up, the model forward as a chain of kernel launches, and the host
 // loops of Ouroboros and of plain greedy decoding.  See include/ouro.h for the contract of each call.
 #include <algorithm>
+#include <atomic>
+#include <chrono>
 #include <cstdio>
 #include <cstring>
 #include <new>
@@ -196,6 +198,7 @@ extern "C" int ouro_create(const ouro_model_desc *t, const ouro_model_mem *tm, c
   auto bail = [&](int code, const std::string &msg) {
     g_create_err = msg;
     if (n->pin) cudaFreeHost(n->pin);
+    if (n->mbox) cudaFreeHost(n->mbox);
     for (auto &e : n->ev) if (e) cudaEventDestroy(e);
     ouro_fast_teardown(n);
     delete n;
@@ -203,6 +206,17 @@ extern "C" int ouro_create(const ouro_model_desc *t, const ouro_model_mem *tm, c
   };
   cudaError_t e = cudaMallocHost((void **)&n->pin, PIN_INTS * sizeof(int32_t));
   if (e != cudaSuccess) return bail(OURO_ENOMEM, std::string("cudaMallocHost: ") + cudaGetErrorString(e));
+  // the mailbox is optional: without mapped host memory the results come back by copy
+  if (cudaHostAlloc((void **)&n->mbox, MBOX_INTS * sizeof(int32_t), cudaHostAllocMapped) == cudaSuccess) {
+    memset(n->mbox, 0, MBOX_INTS * sizeof(int32_t));
+    if (cudaHostGetDevicePointer((void **)&n->mbox_dev, n->mbox, 0) != cudaSuccess) {
+      cudaFreeHost(n->mbox);
+      n->mbox = n->mbox_dev = nullptr;
+    }
+  } else {
+    n->mbox = nullptr;
+    (void)cudaGetLastError();
+  }
   for (auto &ev : n->ev)
     if ((e = cudaEventCreate(&ev)) != cudaSuccess) return bail(OURO_ECUDA, std::string("cudaEventCreate: ") + cudaGetErrorString(e));
   for (int w = 0; w < 2; ++w)
@@ -224,6 +238,7 @@ extern "C" int ouro_destroy(ouro_ctx *c) {
   if (!c) return OURO_EINVAL;
   cudaStreamSynchronize(c->stream);
   if (c->pin) cudaFreeHost(c->pin);
+  if (c->mbox) cudaFreeHost(c->mbox);
   for (auto &e : c->ev) if (e) cudaEventDestroy(e);
   for (auto &e : c->prof_ev) cudaEventDestroy(e);
   ouro_fast_teardown(c);
@@ -295,20 +310,46 @@ extern "C" int ouro_assemble_causal(ouro_ctx *c, int which, const int32_t *token
   return OURO_OK;
 }
 
+// Waits for a kernel to post sequence number `seq` in a mailbox slot.  The wait is bounded: after two seconds
+// the stream is synchronised instead, which also surfaces a launch or execution error.
+static int mbox_wait(ouro_ctx *c, int slot, int32_t seq) {
+  volatile int32_t *flag = c->mbox + slot;
+  const auto t0 = std::chrono::steady_clock::now();
+  for (uint32_t spin = 0; *flag != seq; ++spin) {
+    if ((spin & 4095) == 4095 && std::chrono::steady_clock::now() - t0 > std::chrono::seconds(2)) {
+      CK(cudaStreamSynchronize(c->stream));
+      if (*flag != seq) return fail(c, OURO_ECUDA, "a kernel finished without posting its result");
+      break;
+    }
+  }
+  std::atomic_thread_fence(std::memory_order_acquire);
+  return OURO_OK;
+}
+
 extern "C" int ouro_assemble_candidates(ouro_ctx *c, const int32_t *draft_dev, const int32_t *suffix_dev,
                                         const int32_t *count_dev) {
   if (!c || !draft_dev || ((suffix_dev == nullptr) != (count_dev == nullptr))) return OURO_EINVAL;
   ModelRt &M = c->m[OURO_TARGET];
   const int gamma = c->p.gamma, S = c->p.beta - 1, K = c->p.K;
   if (M.L + 1 + gamma + K * S > M.d.max_seq) return fail(c, OURO_ECAPACITY, "cache length + block rows exceeds max_seq");
-  if (!suffix_dev)
-    launch_lookup_assemble(c->pool, M.blk, c->st, draft_dev, c->cand_suffix, c->cand_count, M.L, gamma, S, K, c->stream);
-  else
-    launch_assemble_candidates(M.blk, c->st, draft_dev, suffix_dev, count_dev, M.L, gamma, S, K, c->stream);
-  CKL();
-  CK(cudaMemcpyAsync(c->pin, &c->st->n_rows, sizeof(int32_t), cudaMemcpyDeviceToHost, c->stream));
-  CK(cudaStreamSynchronize(c->stream));
-  M.blk_rows = c->pin[0];
+  if (!suffix_dev && c->mbox) {
+    const int32_t seq = ++c->mseq;
+    launch_lookup_assemble(c->pool, M.blk, c->st, draft_dev, c->cand_suffix, c->cand_count, M.L, gamma, S, K, c->mbox_dev, seq,
+                           c->stream);
+    CKL();
+    TRY(mbox_wait(c, MBOX_ROWS, seq));
+    M.blk_rows = c->mbox[MBOX_ROWS + 1];
+  } else {
+    if (!suffix_dev)
+      launch_lookup_assemble(c->pool, M.blk, c->st, draft_dev, c->cand_suffix, c->cand_count, M.L, gamma, S, K, nullptr, 0,
+                             c->stream);
+    else
+      launch_assemble_candidates(M.blk, c->st, draft_dev, suffix_dev, count_dev, M.L, gamma, S, K, c->stream);
+    CKL();
+    CK(cudaMemcpyAsync(c->pin, &c->st->n_rows, sizeof(int32_t), cudaMemcpyDeviceToHost, c->stream));
+    CK(cudaStreamSynchronize(c->stream));
+    M.blk_rows = c->pin[0];
+  }
   M.blk_L = M.L;
   M.blk_is_candidate = true;
   return OURO_OK;
@@ -546,13 +587,24 @@ static int accept_step(ouro_ctx *c, const int32_t *argmax_dev, AcceptOut *r) {
     return fail(c, OURO_ESTATE, "no verified candidate block for the current cache length");
   const int gamma = c->p.gamma, S = c->p.beta - 1, L = T.L;
   cudaStream_t s = c->stream;
-  launch_accept_compact_harvest(T.blk, c->st, c->pool, argmax_dev, c->seq_dev, T.d, T.k_cache, T.v_cache, L, gamma, S,
-                                c->p.flags, s);
-  CKL();
   static_assert(sizeof(AcceptOut) <= PIN_INTS * 4, "pinned staging too small");
-  CK(cudaMemcpyAsync(c->pin, &c->st->A, sizeof(AcceptOut), cudaMemcpyDeviceToHost, s));
-  CK(cudaStreamSynchronize(s));
-  memcpy(r, c->pin, sizeof(AcceptOut));
+  static_assert(sizeof(AcceptOut) == (4 + OURO_MAX_GAMMA + OURO_MAX_BETA + 1) * 4 && MBOX_ACCEPT + 1 + sizeof(AcceptOut) / 4 <= MBOX_INTS,
+                "acceptance record and mailbox slot disagree");
+  if (c->mbox) {
+    const int32_t seq = ++c->mseq;
+    launch_accept_compact_harvest(T.blk, c->st, c->pool, argmax_dev, c->seq_dev, T.d, T.k_cache, T.v_cache, L, gamma, S,
+                                  c->p.flags, c->mbox_dev, seq, s);
+    CKL();
+    TRY(mbox_wait(c, MBOX_ACCEPT, seq));
+    memcpy(r, c->mbox + MBOX_ACCEPT + 1, sizeof(AcceptOut));
+  } else {
+    launch_accept_compact_harvest(T.blk, c->st, c->pool, argmax_dev, c->seq_dev, T.d, T.k_cache, T.v_cache, L, gamma, S,
+                                  c->p.flags, nullptr, 0, s);
+    CKL();
+    CK(cudaMemcpyAsync(c->pin, &c->st->A, sizeof(AcceptOut), cudaMemcpyDeviceToHost, s));
+    CK(cudaStreamSynchronize(s));
+    memcpy(r, c->pin, sizeof(AcceptOut));
+  }
   if (r->status != 0) return fail(c, OURO_ETIMEOUT, "device status word " + std::to_string(r->status));
   if (r->n_acc < 1 || r->n_acc > gamma + S + 1) return fail(c, OURO_ECUDA, "acceptance returned an impossible count");
   c->seq.insert(c->seq.end(), r->accepted, r->accepted + r->n_acc);
@@ -688,6 +740,7 @@ extern "C" int ouro_generate(ouro_ctx *c, const int32_t *prompt, int32_t n_promp
     AcceptOut r;
     TRY(accept_step(c, c->a.argmax, &r));
     float ms = 0.f;
+    CK(cudaEventSynchronize(c->ev[4]));               // reached long ago; makes the runtime see it as complete
     CK(cudaEventElapsedTime(&ms, c->ev[1], c->ev[2]));
     st.ms_draft += ms;
     CK(cudaEventElapsedTime(&ms, c->ev[3], c->ev[4]));

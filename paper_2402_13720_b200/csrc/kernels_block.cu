@@ -196,14 +196,25 @@ __global__ void assemble_candidates_kernel(BlockDev b, DevState *st, const int32
 }
 
 // Lookup with key d_gamma (warp 0) and packing in one launch.
+// Writes a result the host is polling for: payload first, then (system-wide fence between) the sequence number.
+__device__ __forceinline__ void mbox_post(int32_t *slot, const int32_t *payload, int n, int32_t seq) {
+  for (int i = 0; i < n; ++i) slot[1 + i] = payload[i];
+  __threadfence_system();
+  *(volatile int32_t *)slot = seq;
+}
+
 __global__ void lookup_assemble_kernel(PoolDev P, BlockDev b, DevState *st, const int32_t *draft, int32_t *suffix,
-                                       int32_t *count, int L, int gamma, int S, int K) {
+                                       int32_t *count, int L, int gamma, int S, int K, int32_t *mbox, int32_t seq) {
   if (threadIdx.x < 32) {
     int32_t key = draft[gamma - 1];
     int n = (key < 0 || P.S == 0) ? 0 : pool_lookup(P, key, K, suffix);
     if (threadIdx.x == 0) *count = n;
   }
   __syncthreads();
+  if (mbox && threadIdx.x == 0) {                       // the row count goes out before the rows are packed
+    const int32_t B = 1 + gamma + (S > 0 ? min(*count, K) : 0) * S;
+    mbox_post(mbox + MBOX_ROWS, &B, 1, seq);
+  }
   assemble_candidates_body(b, st, draft, suffix, count, L, gamma, S, K);
 }
 
@@ -228,9 +239,9 @@ void launch_assemble_candidates(const BlockDev &b, DevState *st, const int32_t *
   assemble_candidates_kernel<<<1, OURO_MAX_ROWS, 0, s>>>(b, st, draft, suffix, count, L, gamma, S, K);
 }
 void launch_lookup_assemble(const PoolDev &P, const BlockDev &b, DevState *st, const int32_t *draft, int32_t *suffix,
-                            int32_t *count, int L, int gamma, int S, int K, cudaStream_t s) {
+                            int32_t *count, int L, int gamma, int S, int K, int32_t *mbox, int32_t seq, cudaStream_t s) {
   OURO_COUNT_LAUNCH();
-  lookup_assemble_kernel<<<1, OURO_MAX_ROWS, 0, s>>>(P, b, st, draft, suffix, count, L, gamma, S, K);
+  lookup_assemble_kernel<<<1, OURO_MAX_ROWS, 0, s>>>(P, b, st, draft, suffix, count, L, gamma, S, K, mbox, seq);
 }
 void launch_assemble_causal(const BlockDev &b, const int32_t *tokens, int n, int L, cudaStream_t s) {
   OURO_COUNT_LAUNCH();
@@ -377,9 +388,12 @@ __global__ void harvest_kernel(BlockDev b, DevState *st, PoolDev P, const int32_
 // waiting for block 0, then moves its cache row if the row belongs to the accepted suffix.
 __global__ void accept_compact_harvest_kernel(BlockDev b, DevState *st, PoolDev P, const int32_t *o, int32_t *seq_dev,
                                               unsigned char *k_cache, unsigned char *v_cache, int L, int gamma, int S,
-                                              int max_seq, int row_bytes, unsigned flags) {
+                                              int max_seq, int row_bytes, unsigned flags, int32_t *mbox, int32_t seq) {
   if (blockIdx.x == 0) {
-    if (threadIdx.x == 0) accept_body(b, st, o, seq_dev, gamma, S);
+    if (threadIdx.x == 0) {
+      accept_body(b, st, o, seq_dev, gamma, S);
+      if (mbox) mbox_post(mbox + MBOX_ACCEPT, &st->A, 4 + OURO_MAX_GAMMA + OURO_MAX_BETA + 1, seq);   // A .. status
+    }
     __syncthreads();
     if (threadIdx.x < 32 && (flags & (OURO_HARVEST_MATCHED | OURO_HARVEST_CANDIDATES | OURO_HARVEST_ACCEPTED)))
       harvest_body(b, st, P, o, seq_dev, gamma, S, flags);
@@ -410,12 +424,12 @@ __global__ void accept_compact_harvest_kernel(BlockDev b, DevState *st, PoolDev 
 
 void launch_accept_compact_harvest(const BlockDev &b, DevState *st, const PoolDev &P, const int32_t *o, int32_t *seq_dev,
                                    const ouro_model_desc &d, void *k_cache, void *v_cache, int L, int gamma, int S,
-                                   unsigned flags, cudaStream_t s) {
+                                   unsigned flags, int32_t *mbox, int32_t seq, cudaStream_t s) {
   OURO_COUNT_LAUNCH();
   const int es = d.dtype == OURO_BF16 ? 2 : 4;
   accept_compact_harvest_kernel<<<1 + S * d.n_layers * 2, 128, 0, s>>>(b, st, P, o, seq_dev, (unsigned char *)k_cache,
                                                                       (unsigned char *)v_cache, L, gamma, S, d.max_seq,
-                                                                      d.n_kv_heads * d.head_dim * es, flags);
+                                                                      d.n_kv_heads * d.head_dim * es, flags, mbox, seq);
 }
 
 // ------------------------------------------------------------- phrase-level drafting (Section 3.1)

@@ -119,6 +119,10 @@ struct ouro_ctx {
   // host side
   std::vector<int32_t> seq;       // the text: prompt + accepted tokens (last one pending)
   int32_t *pin = nullptr;         // pinned host staging (PIN_INTS ints)
+  // Mailbox in mapped pinned memory: the two results the host needs in every step (block row count, acceptance
+  // record) are written there by the kernels themselves, payload first, then a sequence number the host polls.
+  int32_t *mbox = nullptr, *mbox_dev = nullptr;
+  int32_t mseq = 0;
   ouro_drafter_fn drafter = nullptr;
   void *drafter_user = nullptr;
   int32_t step = 0;
@@ -157,10 +161,11 @@ void launch_compact(const ouro_model_desc &d, void *k_cache, void *v_cache, cons
 void launch_harvest(const BlockDev &b, DevState *st, const PoolDev &P, const int32_t *o, const int32_t *seq_dev,
                     int gamma, int S, unsigned flags, cudaStream_t s);
 void launch_lookup_assemble(const PoolDev &P, const BlockDev &b, DevState *st, const int32_t *draft, int32_t *suffix,
-                            int32_t *count, int L, int gamma, int S, int K, cudaStream_t s);
+                            int32_t *count, int L, int gamma, int S, int K, int32_t *mbox, int32_t seq, cudaStream_t s);
 void launch_accept_compact_harvest(const BlockDev &b, DevState *st, const PoolDev &P, const int32_t *o, int32_t *seq_dev,
                                    const ouro_model_desc &d, void *k_cache, void *v_cache, int L, int gamma, int S,
-                                   unsigned flags, cudaStream_t s);
+                                   unsigned flags, int32_t *mbox, int32_t seq, cudaStream_t s);
+enum { MBOX_INTS = 128, MBOX_ROWS = 0, MBOX_ACCEPT = 16 };   // [flag, rows] and [flag, acceptance record] slots
 void launch_draft_lookup_assemble(const PoolDev &P, const BlockDev &b, DevState *st, const int32_t *tokens, int n,
                                   int32_t *suffix, int32_t *count, int L, int S, int K, cudaStream_t s);
 void launch_draft_accept_compact(const BlockDev &b, DevState *st, const int32_t *o, int32_t *out_dev, int have, int gamma,
