@@ -607,3 +607,26 @@ def test_phrase_level_drafting_bf16_self_draft():
         eng.close()
     assert res[0]["target_calls"] == res[1]["target_calls"] and res[0]["full_accepts"] == res[0]["target_calls"]
     assert res[1]["draft_calls"] <= res[0]["draft_calls"] == 4 * res[0]["target_calls"]
+
+
+def test_phrase_level_drafting_edge_cases():
+    """Long catch-up (the uncached text does not fit one block beside the candidates), K = 0 (every round is a plain
+    single-token forward) and beta = 1 (phrases have no suffix): the drafts stay those of token-level drafting."""
+    import dataclasses
+    w = synth.model_weights(TINY, 2, device="cuda:0")
+    prompt = synth.prompt(2, TINY.vocab, 125, 0.5, 4, 8)             # 125 + K*S rows > OURO_MAX_ROWS on the first round
+    for gamma, beta, K in ((3, 4, 4), (3, 4, 0), (2, 1, 3)):
+        P0 = synth.DecodeParams(gamma, beta, K, 8, 4)
+        P1 = dataclasses.replace(P0, draft_phrases=True)
+        outs = []
+        for P in (P0, P1):
+            eng = binding.Engine(TINY, w, P, TINY, w)
+            van, _ = eng.generate_vanilla(prompt, 20)
+            out, st = eng.generate(prompt, 20)
+            assert np.array_equal(out, van)
+            outs.append(st)
+            eng.close()
+        assert outs[0]["target_calls"] == outs[1]["target_calls"]
+        assert outs[1]["draft_calls"] <= outs[0]["draft_calls"]
+        if K == 0 or beta == 1:
+            assert outs[1]["draft_calls"] == outs[0]["draft_calls"]
