@@ -377,7 +377,8 @@ __global__ void __launch_bounds__(THREADS) attn_span_kernel(const AttnParams p) 
   }
 }
 
-// Folds a row's spans in ascending order and normalises.  One warp per (row, head).
+// Folds a row's spans and normalises.  One warp per (row, head).  First the largest span maximum, then one
+// weighted sum over the spans in ascending order: the loads of different spans do not wait for one another.
 template <int HD>
 __global__ void attn_merge_kernel(const AttnParams p) {
   constexpr int PW = HD + 2, DPL = HD / 32;
@@ -389,17 +390,21 @@ __global__ void attn_merge_kernel(const AttnParams p) {
   const int nv = p.lin_end[r] + p.seg_len[r];
   const int ns = (nv + SPAN - 1) / SPAN;
   const float *src = p.part + ((size_t)r * p.H + head) * p.cap * PW;
-  float m = -INFINITY, l = 0.f, acc[DPL];
+  float mx = -INFINITY;
+  for (int c = lane; c < ns; c += 32) mx = fmaxf(mx, src[(size_t)c * PW]);
+#pragma unroll
+  for (int o = 16; o; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+  float l = 0.f, acc[DPL];
 #pragma unroll
   for (int i = 0; i < DPL; ++i) acc[i] = 0.f;
+#pragma unroll 4
   for (int c = 0; c < ns; ++c) {
     const float *pc = src + (size_t)c * PW;
-    const float mp = pc[0], mn = fmaxf(m, mp);
-    const float a = (m == -INFINITY) ? 0.f : exp2f(m - mn), b = (mp == -INFINITY) ? 0.f : exp2f(mp - mn);
-    l = l * a + pc[1] * b;
+    const float mp = pc[0];
+    const float w = (mp == -INFINITY) ? 0.f : exp2f(mp - mx);     // mx is finite: the first span holds a visible key
+    l += pc[1] * w;
 #pragma unroll
-    for (int i = 0; i < DPL; ++i) acc[i] = acc[i] * a + pc[2 + lane + 32 * i] * b;
-    m = mn;
+    for (int i = 0; i < DPL; ++i) acc[i] += pc[2 + lane + 32 * i] * w;
   }
   const float inv = 1.0f / l;
 #pragma unroll

@@ -155,6 +155,16 @@ __device__ __forceinline__ void tmem_ld_wait32(float *v) {
                :
                : "memory");
 }
+// 16 columns, issued and waited for.
+__device__ __forceinline__ void tmem_ld16(uint32_t addr, float *v) {
+  asm volatile("tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+               : "=f"(v[0]), "=f"(v[1]), "=f"(v[2]), "=f"(v[3]), "=f"(v[4]), "=f"(v[5]), "=f"(v[6]), "=f"(v[7]), "=f"(v[8]), "=f"(v[9]), "=f"(v[10]), "=f"(v[11]), "=f"(v[12]), "=f"(v[13]), "=f"(v[14]), "=f"(v[15])
+               : "r"(addr));
+  asm volatile("tcgen05.wait::ld.sync.aligned;"
+               : "+f"(v[0]), "+f"(v[1]), "+f"(v[2]), "+f"(v[3]), "+f"(v[4]), "+f"(v[5]), "+f"(v[6]), "+f"(v[7]), "+f"(v[8]), "+f"(v[9]), "+f"(v[10]), "+f"(v[11]), "+f"(v[12]), "+f"(v[13]), "+f"(v[14]), "+f"(v[15])
+               :
+               : "memory");
+}
 __device__ __forceinline__ void fence_before_sync() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void fence_after_sync() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
@@ -474,9 +484,12 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tm_kernel(const __grid_consta
         const int nk = active ? min(nv - c0, CH) : 0;  // keys of this chunk the row sees: tile columns below nk
         const int nk_w = __reduce_max_sync(0xffffffffu, nk);
         const bool whole = __all_sync(0xffffffffu, !active || nk >= CH);   // no score of an active row is masked
-        if (nk_w > 0) {                                // TMEM loads are warp-wide: every lane takes part
-          // a half of the chunk that no row of the warp reaches takes no arithmetic (its scores are read all the same)
-          const bool need_own = h * 64 < nk_w;
+        // Both forms below compute the same numbers for a row, in the same order (four interleaved partial sums
+        // over ascending keys; a masked key adds an exact zero), so which one a warp takes - that depends on its
+        // other rows - never shows in a row's result.  TMEM loads are warp-wide: every lane takes part in them.
+        uint8_t *prow = smem + OFF_P + b * TILE + h * HALF + t * 128;     // this thread's 128 bytes of P
+        float mn = m_run, sum = 0.f;
+        if (whole) {
           // ---- row maximum over the chunk (scaling by a positive factor commutes with max, bit for bit)
           float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
@@ -486,59 +499,75 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tm_kernel(const __grid_consta
             tmem_ld32_issue(lane_addr + b * 128 + hh * 64 + 32, vm + 32);
             tmem_ld_wait32(vm);
             tmem_ld_wait32(vm + 32);
-            if (whole) {
 #pragma unroll
-              for (int j = 0; j < 64; ++j) mx4[j & 3] = fmaxf(mx4[j & 3], vm[j]);
-            } else if (hh * 64 < nk_w) {
-#pragma unroll
-              for (int j = 0; j < 64; ++j)
-                if (hh * 64 + j < nk) mx4[j & 3] = fmaxf(mx4[j & 3], vm[j]);
-            }
+            for (int j = 0; j < 64; ++j) mx4[j & 3] = fmaxf(mx4[j & 3], vm[j]);
           }
-          const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
-          const float mn = fmaxf(m_run, mx * p.scale_log2);   // finite for an active row: it sees key c0 at least
+          mn = fmaxf(m_run, fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * p.scale_log2);
           // ---- P = exp2(S - max) for this thread's 64 keys
           float v[64];
           tmem_ld32_issue(lane_addr + b * 128 + h * 64, v);
           tmem_ld32_issue(lane_addr + b * 128 + h * 64 + 32, v + 32);
           tmem_ld_wait32(v);
           tmem_ld_wait32(v + 32);
-          float sum = 0.f;
-          uint8_t *prow = smem + OFF_P + b * TILE + h * HALF + t * 128;   // this thread's 128 bytes of P
-          if (active && need_own) {
-            float sum4[4] = {0.f, 0.f, 0.f, 0.f};      // four interleaved partial sums, folded in a fixed order
+          if (active) {
+            float sum4[4] = {0.f, 0.f, 0.f, 0.f};
             uint32_t w[32];
-            if (whole) {
 #pragma unroll
-              for (int j = 0; j < 64; j += 2) {
-                const float p0 = ex2(v[j] * p.scale_log2 - mn), p1 = ex2(v[j + 1] * p.scale_log2 - mn);
-                sum4[j & 3] += p0;
-                sum4[(j & 3) + 1] += p1;
-                w[j >> 1] = pack_bf16(p0, p1);
-              }
-            } else {
-#pragma unroll
-              for (int j = 0; j < 64; j += 2) {
-                const float p0 = (h * 64 + j < nk) ? ex2(v[j] * p.scale_log2 - mn) : 0.f;
-                const float p1 = (h * 64 + j + 1 < nk) ? ex2(v[j + 1] * p.scale_log2 - mn) : 0.f;
-                sum4[j & 3] += p0;
-                sum4[(j & 3) + 1] += p1;
-                w[j >> 1] = pack_bf16(p0, p1);
-              }
+            for (int j = 0; j < 64; j += 2) {
+              const float p0 = ex2(v[j] * p.scale_log2 - mn), p1 = ex2(v[j + 1] * p.scale_log2 - mn);
+              sum4[j & 3] += p0;
+              sum4[(j & 3) + 1] += p1;
+              w[j >> 1] = pack_bf16(p0, p1);
             }
             sum = (sum4[0] + sum4[1]) + (sum4[2] + sum4[3]);
 #pragma unroll
             for (int q8 = 0; q8 < 8; ++q8)              // 16-byte piece q8 of key half h: keys 64 h + 8 q8 ..
               *reinterpret_cast<uint4 *>(prow + ((q8 ^ (t & 7)) << 4)) = make_uint4(w[4 * q8], w[4 * q8 + 1], w[4 * q8 + 2], w[4 * q8 + 3]);
-          } else if (active) {
+          }
+        } else if (nk_w > 0) {
+          // a chunk that ends inside the block's own keys: only the 16-key pieces below nk_w are looked at
+          const int npc = (nk_w + 15) >> 4;
+          float mxv = -INFINITY;
+          for (int pc = 0; pc < npc; ++pc) {
+            float v[16];
+            tmem_ld16(lane_addr + b * 128 + pc * 16, v);
 #pragma unroll
-            for (int q8 = 0; q8 < 8; ++q8) *reinterpret_cast<uint4 *>(prow + (q8 << 4)) = make_uint4(0u, 0u, 0u, 0u);
+            for (int j = 0; j < 16; ++j)
+              if (pc * 16 + j < nk) mxv = fmaxf(mxv, v[j]);
           }
-          if (active) {
-            alpha = (m_run == -INFINITY) ? 0.f : ex2(m_run - mn);
-            l_run = l_run * alpha + sum;
-            m_run = mn;
+          mn = fmaxf(m_run, mxv * p.scale_log2);       // finite for an active row: it sees key c0 at least
+          float sum4[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+          for (int q = 0; q < 4; ++q) {                 // the four 16-key pieces of this thread's half
+            const int pc = 4 * h + q;
+            uint32_t w[8];
+#pragma unroll
+            for (int j = 0; j < 8; ++j) w[j] = 0u;
+            if (pc < npc) {
+              float v[16];
+              tmem_ld16(lane_addr + b * 128 + pc * 16, v);
+              if (active) {
+#pragma unroll
+                for (int j = 0; j < 16; j += 2) {
+                  const float p0 = (pc * 16 + j < nk) ? ex2(v[j] * p.scale_log2 - mn) : 0.f;
+                  const float p1 = (pc * 16 + j + 1 < nk) ? ex2(v[j + 1] * p.scale_log2 - mn) : 0.f;
+                  sum4[j & 3] += p0;
+                  sum4[(j & 3) + 1] += p1;
+                  w[j >> 1] = pack_bf16(p0, p1);
+                }
+              }
+            }
+            if (active) {
+              *reinterpret_cast<uint4 *>(prow + (((2 * q) ^ (t & 7)) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
+              *reinterpret_cast<uint4 *>(prow + (((2 * q + 1) ^ (t & 7)) << 4)) = make_uint4(w[4], w[5], w[6], w[7]);
+            }
           }
+          sum = (sum4[0] + sum4[1]) + (sum4[2] + sum4[3]);
+        }
+        if (active) {
+          alpha = (m_run == -INFINITY) ? 0.f : ex2(m_run - mn);
+          l_run = l_run * alpha + sum;
+          m_run = mn;
         }
         fence_async_smem();
         fence_before_sync();
