@@ -332,11 +332,11 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tm_kernel(const __grid_consta
   if (n_items > 0) {
     if (warp == 0) {
       // ================================================================ tile producer (TMA; whole warp for the patches)
-      bool ok = true;
+      // (a wait that gives up raises the abort flag and the status word itself; nobody blocks after that)
       for (int i = 0; i < n_items; ++i) {
         const int it = ms->items[i], ci = it & 7, go = (it >> 3) & 63, st = i & 1;
         if (i >= early) {
-          if (i >= 2) ok = mbar_wait(&ms->empty[st], ((i >> 1) - 1) & 1, ms, p.status) && ok;
+          if (i >= 2) mbar_wait(&ms->empty[st], ((i >> 1) - 1) & 1, ms, p.status);
           if (lane == 0) {
             if (it & IT_REUSE) mbar_arrive(&ms->full[st]);   // nothing to fetch: the phase completes at once
             else request_tile(i, ci);
@@ -344,7 +344,7 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tm_kernel(const __grid_consta
         }
         if (it & IT_PATCH) {
           // a candidate's pass: its suffix rows go over the tile the TMA fetched (slots = positions up to the trunk)
-          ok = mbar_wait(&ms->full[st], (i >> 1) & 1, ms, p.status) && ok;
+          mbar_wait(&ms->full[st], (i >> 1) & 1, ms, p.status);
           const int c0 = span0 + ci * CH, last = ms->gs[go + 1] - 1;
           const int lin_g = ms->lin[last], seg_g = p.seg_start[last], len_g = ms->len[last];
           const int lo = max(c0, lin_g), hi = min(c0 + CH, lin_g + len_g);
@@ -372,7 +372,7 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tm_kernel(const __grid_consta
     } else if (warp == 1) {
       // ================================================================ contraction issue
       if (lane == 0) {
-        bool ok = true, issued = false;
+        bool issued = false;
         uint32_t patch_par = 0;                        // bit st: parity of the next patched tile of stage st
         auto issue_s = [&](int i) {
           const uint64_t da = desc_k(sm_u + OFF_Q), db = desc_k(sm_u + OFF_K + (i & 1) * TILE);
@@ -404,7 +404,6 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tm_kernel(const __grid_consta
             }
             if (!ready) {
               if (atomicExch(&ms->abort_flag, 1) == 0) atomicExch(p.status, 1);
-              ok = false;
             }
             tile_taken(i);
             fence_after_sync();
@@ -426,7 +425,6 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tm_kernel(const __grid_consta
           }
           if (!p_done) {
             if (atomicExch(&ms->abort_flag, 1) == 0) atomicExch(p.status, 1);
-            ok = false;
           }
           fence_after_sync();
           {
@@ -455,10 +453,10 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tm_kernel(const __grid_consta
       float o_reg[HD / 2];
 #pragma unroll
       for (int i = 0; i < HD / 2; ++i) o_reg[i] = 0.f;
-      bool ok = true, pending = false, act_prev = false;
+      bool pending = false, act_prev = false;
 
       auto accumulate = [&](int i) {                   // O = O * alpha + O_c of pass i
-        ok = mbar_wait(&ms->o_ready[i & 1], (i >> 1) & 1, ms, p.status) && ok;
+        mbar_wait(&ms->o_ready[i & 1], (i >> 1) & 1, ms, p.status);
         fence_after_sync();
         if (__any_sync(0xffffffffu, act_prev)) {        // TMEM loads are warp-wide: every lane takes part
           float v[64];
@@ -478,7 +476,7 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tm_kernel(const __grid_consta
         const int it = ms->items[i], ci = it & 7, go = (it >> 3) & 63, b = i & 1;
         const int c0 = span0 + ci * CH;
         const bool active = has && nv > c0 && (go == 63 || go == my_o);
-        ok = mbar_wait(&ms->s_ready[b], (i >> 1) & 1, ms, p.status) && ok;
+        mbar_wait(&ms->s_ready[b], (i >> 1) & 1, ms, p.status);
         fence_after_sync();
         float alpha = 1.f;
         const int nk = active ? min(nv - c0, CH) : 0;  // keys of this chunk the row sees: tile columns below nk
