@@ -40,6 +40,7 @@ struct AttnParams {
   float scale_log2;
   float *part;                     // [rows][H][cap][HD+2]: max (log2 domain), sum, unnormalised output
   __nv_bfloat16 *out;              // [rows][H*HD]
+  int direct;                      // every row's keys lie in span 0: the span kernel normalises and writes `out` itself
 };
 
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -366,6 +367,17 @@ __global__ void __launch_bounds__(THREADS) attn_span_kernel(const AttnParams p) 
 #pragma unroll
     for (int i = 0; i < 2 * MT; ++i) {
       if (nv[i] <= span0) continue;
+      if (p.direct) {
+        // what the merge kernel would compute from this single span: weight exp2(0) = 1, then o * (1 / l)
+        const float inv = 1.0f / l_run[i];
+#pragma unroll
+        for (int nt = 0; nt < NT2; ++nt) {
+          int d = warp * DW + 8 * nt + 2 * (lane & 3);
+          *reinterpret_cast<__nv_bfloat162 *>(p.out + ((size_t)rr[i] * p.H + hh[i]) * HD + d) =
+              __floats2bfloat162_rn(o[i >> 1][nt][2 * (i & 1)] * inv, o[i >> 1][nt][2 * (i & 1) + 1] * inv);
+        }
+        continue;
+      }
       float *dst = p.part + (((size_t)rr[i] * p.H + hh[i]) * p.cap + sc) * PW;
       if (warp == 0 && (lane & 3) == 0) { dst[0] = m_run[i]; dst[1] = l_run[i]; }
 #pragma unroll
@@ -449,7 +461,6 @@ void launch_attention_merge(const ouro_model_desc &d, const BlockDev &b, int row
 void launch_attention_tc(const ouro_model_desc &d, const void *q, const void *k_cache, const void *v_cache, const BlockDev &b,
                          int rows, int L, int n_vis_max, int layer, float *part, void *out, cudaStream_t s) {
   OURO_COUNT_LAUNCH();
-  OURO_COUNT_LAUNCH();
   AttnParams p;
   size_t off = (size_t)layer * d.max_seq * d.n_kv_heads * d.head_dim;
   p.q = (const __nv_bfloat16 *)q;
@@ -463,11 +474,13 @@ void launch_attention_tc(const ouro_model_desc &d, const void *q, const void *k_
   p.out = (__nv_bfloat16 *)out;
   const int m_all = (d.n_heads / d.n_kv_heads) * rows;      // query rows per kv head, served 64 per CTA
   dim3 grid((n_vis_max + SPAN - 1) / SPAN, d.n_kv_heads, (m_all + QR - 1) / QR), mgrid(rows, (d.n_heads + 3) / 4);
+  p.direct = n_vis_max <= SPAN;                             // a single span: nothing to fold, no second launch
+  if (!p.direct) OURO_COUNT_LAUNCH();
   if (d.head_dim == 128) {
     launch_pdl(attn_span_kernel<128>, grid, THREADS, Smem<128>::BYTES, s, p);
-    launch_pdl(attn_merge_kernel<128>, mgrid, 128, 0, s, p);
+    if (!p.direct) launch_pdl(attn_merge_kernel<128>, mgrid, 128, 0, s, p);
   } else {
     launch_pdl(attn_span_kernel<64>, grid, THREADS, Smem<64>::BYTES, s, p);
-    launch_pdl(attn_merge_kernel<64>, mgrid, 128, 0, s, p);
+    if (!p.direct) launch_pdl(attn_merge_kernel<64>, mgrid, 128, 0, s, p);
   }
 }

@@ -79,6 +79,8 @@ struct TmParams {
   int n_spans;
   float scale_log2;
   float *part;                     // [rows][H][cap][HD+2]: max (log2 domain), sum, unnormalised output
+  __nv_bfloat16 *out;              // [rows][H*HD], written here only when `direct`
+  int direct;                      // every row's keys lie in span 0: normalise and write `out`, no folding needed
   int *status;
 };
 
@@ -578,11 +580,22 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tm_kernel(const __grid_consta
       if (pending) accumulate(n_items - 1);
       // ---- the span's piece of this row: the two halves of the row sum are added in a fixed order
       float *lsum = reinterpret_cast<float *>(smem + OFF_Q);      // Q is no longer read: every contraction has completed
-      if (h == 1) lsum[t] = l_run;
+      lsum[h * QR + t] = l_run;
       asm volatile("bar.sync 1, %0;" ::"n"(ROW_THREADS) : "memory");
-      if (has && nv > span0) {
+      if (has && nv > span0 && p.direct) {
+        // what the merge kernel would compute from this single span: weight exp2(0) = 1, then o * (1 / l)
+        const float inv = 1.0f / (lsum[t] + lsum[QR + t]);
+        __nv_bfloat16 *dst = p.out + ((size_t)r * p.H + kvh * g + hq) * HD + h * 64;
+#pragma unroll
+        for (int d = 0; d < HD / 2; d += 8) {
+          uint32_t w[4];
+#pragma unroll
+          for (int e = 0; e < 4; ++e) w[e] = pack_bf16(o_reg[d + 2 * e] * inv, o_reg[d + 2 * e + 1] * inv);
+          *reinterpret_cast<uint4 *>(dst + d) = make_uint4(w[0], w[1], w[2], w[3]);
+        }
+      } else if (has && nv > span0) {
         float *dst = p.part + (((size_t)r * p.H + kvh * g + hq) * p.cap + sc) * PW;
-        if (h == 0) *reinterpret_cast<float2 *>(dst) = make_float2(m_run, l_run + lsum[t]);
+        if (h == 0) *reinterpret_cast<float2 *>(dst) = make_float2(m_run, lsum[t] + lsum[QR + t]);
 #pragma unroll
         for (int d = 0; d < HD / 2; d += 2) *reinterpret_cast<float2 *>(dst + 2 + h * 64 + d) = make_float2(o_reg[d], o_reg[d + 1]);
       }
@@ -608,10 +621,11 @@ int attention_tm_setup() {
 }
 
 // kmap / vmap: CUtensorMap objects over the whole K and V caches, [n_layers * max_seq][Hkv * 128] bf16 with a
-// 64 x 128 box in 128-byte swizzle.  Launches the span kernel; the caller folds the spans afterwards.
-void launch_attention_tm(const ouro_model_desc &d, const void *q, const void *kmap, const void *vmap, const void *k_cache,
+// 64 x 128 box in 128-byte swizzle.  Launches the span kernel.  Returns true when the spans still have to be folded
+// by the caller (launch_attention_merge); with a single span the kernel has written `out` itself.
+bool launch_attention_tm(const ouro_model_desc &d, const void *q, const void *kmap, const void *vmap, const void *k_cache,
                          const void *v_cache, const BlockDev &b, int rows, int L, int n_vis_max, int layer, float *part,
-                         int *status, cudaStream_t s) {
+                         void *out, int *status, cudaStream_t s) {
   OURO_COUNT_LAUNCH();
   TmParams p;
   p.kmap = *reinterpret_cast<const CUtensorMap *>(kmap);
@@ -626,9 +640,12 @@ void launch_attention_tm(const ouro_model_desc &d, const void *q, const void *km
   p.row0 = layer * d.max_seq;
   p.scale_log2 = 1.4426950408889634f / sqrtf((float)d.head_dim);
   p.part = part;
+  p.out = (__nv_bfloat16 *)out;
+  p.direct = n_vis_max <= SPAN;
   p.status = status;
   const int m_all = (d.n_heads / d.n_kv_heads) * rows;
   p.n_spans = (n_vis_max + SPAN - 1) / SPAN;
   dim3 grid(p.n_spans * d.n_kv_heads, (m_all + QR - 1) / QR);
   launch_pdl(attn_tm_kernel, grid, THREADS, SMEM_BYTES, s, p);
+  return !p.direct;
 }

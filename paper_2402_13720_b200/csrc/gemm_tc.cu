@@ -1021,9 +1021,9 @@ int ouro_fast_layer(ouro_ctx *c, int which, int l, int rows) {
   {
     ProfScope ps(c, OURO_PROF_ATTENTION);
     if (c->fast->s.m[which].kv_maps) {
-      launch_attention_tm(d, a.q, &c->fast->s.m[which].kmap, &c->fast->s.m[which].vmap, M.k_cache, M.v_cache, M.blk, rows, M.L,
-                          M.L + rows, l, c->fast->s.attn_part, &c->st->status, s);
-      launch_attention_merge(d, M.blk, rows, c->fast->s.attn_part, a.att, s);
+      if (launch_attention_tm(d, a.q, &c->fast->s.m[which].kmap, &c->fast->s.m[which].vmap, M.k_cache, M.v_cache, M.blk, rows,
+                              M.L, M.L + rows, l, c->fast->s.attn_part, a.att, &c->st->status, s))
+        launch_attention_merge(d, M.blk, rows, c->fast->s.attn_part, a.att, s);
     } else if (attention_tc_supported(d))
       launch_attention_tc(d, a.q, M.k_cache, M.v_cache, M.blk, rows, M.L, M.L + rows, l, c->fast->s.attn_part, a.att, s);
     else

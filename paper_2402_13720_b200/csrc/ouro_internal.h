@@ -206,6 +206,6 @@ void launch_attention_merge(const ouro_model_desc &d, const BlockDev &b, int row
 // ---- attn_tm.cu (tcgen05 path, head dim 128) ---------------------------------------------------
 bool attention_tm_supported(const ouro_model_desc &d);
 int attention_tm_setup();
-void launch_attention_tm(const ouro_model_desc &d, const void *q, const void *kmap, const void *vmap, const void *k_cache,
+bool launch_attention_tm(const ouro_model_desc &d, const void *q, const void *kmap, const void *vmap, const void *k_cache,
                          const void *v_cache, const BlockDev &b, int rows, int L, int n_vis_max, int layer, float *part,
-                         int *status, cudaStream_t s);
+                         void *out, int *status, cudaStream_t s);
