@@ -82,7 +82,7 @@ typedef struct {
   const void *const *w_gate;    /* [d_ffn, d_model] */
   const void *const *w_up;      /* [d_ffn, d_model] */
   const void *const *w_down;    /* [d_model, d_ffn] */
-  void *k_cache, *v_cache;
+  void *k_cache, *v_cache;      /* [n_layers, max_seq, n_kv_heads, head_dim]; ouro_create clears them (unused rows must be finite) */
 } ouro_model_mem;
 
 /* gamma: draft length (Eq. 1).  beta: phrase length INCLUDING its first token p_1 = d_gamma (Section

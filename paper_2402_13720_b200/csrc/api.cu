@@ -223,6 +223,16 @@ extern "C" int ouro_create(const ouro_model_desc *t, const ouro_model_mem *tm, c
     if (n->m[w].present)
       launch_rope_table(n->m[w].rope_cos, n->m[w].rope_sin, n->m[w].d.max_seq, n->m[w].d.head_dim, n->m[w].d.rope_theta,
                         n->stream);
+  // The attention kernels multiply masked keys' V rows by an exact zero, so rows nobody has written yet must not
+  // hold NaN or infinity: the caches start out cleared.
+  for (int w = 0; w < 2; ++w)
+    if (n->m[w].present) {
+      const ouro_model_desc &md = n->m[w].d;
+      const size_t bytes = (size_t)md.n_layers * md.max_seq * md.n_kv_heads * md.head_dim * (md.dtype == OURO_BF16 ? 2 : 4);
+      if ((e = cudaMemsetAsync(n->m[w].k_cache, 0, bytes, n->stream)) != cudaSuccess ||
+          (e = cudaMemsetAsync(n->m[w].v_cache, 0, bytes, n->stream)) != cudaSuccess)
+        return bail(OURO_ECUDA, std::string("clearing the KV cache: ") + cudaGetErrorString(e));
+    }
   launch_pool_clear(n->pool, n->st, n->stream);
   launch_set_state(n->st, n->seq_dev, 1, 0, 1, n->stream);
   int rc = ouro_fast_setup(n);
