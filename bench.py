@@ -309,6 +309,44 @@ def run_generate(args, device):
         "ms_draft_per_step": st["ms_draft"] / st["target_calls"], "identical_to_vanilla": bool(np.array_equal(out, van))}
     eng2.close()
 
+    # Sweeps over the method's knobs (the paper's K study, its gamma / beta grid and its component ablation, on
+    # synthetic inputs): replayed drafts at the middle agreement level plus the seeded phrase source, one engine
+    # per setting on the same weights.
+    sweep = {}
+    if args.sweep:
+        def one(Pv, phrases=True):
+            e3 = binding.Engine(T, wt, Pv, D, wd, device=device)
+
+            def drafter(seq, g, step):
+                d = synth.corrupt_drafts(SEED + 7, truth, len(seq), g, T.vocab, 0.12, 0.03, step)
+                if phrases and Pv.K > 0 and Pv.S > 0:
+                    grams = np.empty((Pv.K, Pv.beta), dtype=np.int32)
+                    for j in range(Pv.K):
+                        grams[j, 0] = d[-1]
+                        grams[j, 1:] = synth.corrupt_drafts(SEED + 11 + j, truth, len(seq) + g, Pv.S, T.vocab, 0.08 * (j + 1), 0.0, step)
+                    e3.phrase_update(grams[::-1])
+                return d
+
+            e3.set_drafter(drafter)
+            out, st = e3.generate(prompt, gen)
+            e3.set_drafter(None)
+            e3.close()
+            return {"tokens_per_s": round(len(out) / (st["ms_total"] * 1e-3), 1),
+                    "tokens_per_target_call": round(len(out) / st["target_calls"], 2),
+                    "ms_target_per_call": round(st["ms_target"] / st["target_calls"], 3),
+                    "identical_to_vanilla": bool(np.array_equal(out, van))}
+
+        rp = dataclasses.replace
+        sweep["K"] = {k: one(rp(P, K=k)) for k in (0, 1, 2, 4, 8, 12)}
+        sweep["gamma"] = {g: one(rp(P, gamma=g)) for g in (2, 4, 6, 8, 12)}
+        sweep["beta"] = {b: one(rp(P, beta=b)) for b in (3, 5, 9, 13)}
+        sweep["components"] = {
+            "token-level drafts only (K = 0)": one(rp(P, K=0), phrases=False),
+            "+ phrases from the pool as harvested (no phrase source)": one(P, phrases=False),
+            "+ seeded phrase source": one(P),
+            "paper-pure harvest flags + phrase source": one(P.paper_pure()),
+        }
+
     try:
         peaks = json.load(open(os.path.join(ROOT, "MEASURED_PEAKS.json")))
     except Exception:
@@ -325,6 +363,8 @@ def run_generate(args, device):
             "verify_forward_frac_of_peak": wbytes / (mid["ms_target_per_call"] * 1e-3) / 1e9 / peak,
             "with_phrases_vs_vanilla": res["replay_mid_phrases"]["tokens_per_s"] / res["vanilla"]["tokens_per_s"],
             "results": res}
+    if sweep:
+        line["sweep"] = sweep
     print(json.dumps(line))
     eng.close()
 
@@ -340,6 +380,7 @@ def main():
     ap.add_argument("--generate", default=None, choices=["C1", "C3", "C4", "C5"],
                     help="instead of the verify-step benchmark: whole generation on that configuration "
                          "(vanilla greedy vs Ouroboros, natural and replayed drafts), one JSON line")
+    ap.add_argument("--sweep", action="store_true", help="with --generate: K, gamma, beta and component sweeps as well")
     ap.add_argument("--gen-tokens", type=int, default=0, help="override the configuration's generation length")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", "0"))
