@@ -630,3 +630,43 @@ def test_phrase_level_drafting_edge_cases():
         assert outs[1]["draft_calls"] <= outs[0]["draft_calls"]
         if K == 0 or beta == 1:
             assert outs[1]["draft_calls"] == outs[0]["draft_calls"]
+
+
+# --------------------------------------- tcgen05 attention: GQA, several rounds of query rows, span boundaries
+
+GQAB = synth.ModelDesc(2, 512, 8, 2, 128, 1024, 1000, 1200, "bf16")   # 4 query heads per kv head, head_dim 128
+
+
+@pytest.mark.parametrize("seed,L_prompt", [(0, 40), (1, 509), (2, 1000), (3, 129)])
+def test_verify_logits_bf16_gqa_head_dim_128(seed, L_prompt):
+    """69 block rows x 4 query heads per kv head = 276 query rows (three rounds of 128) with 8 candidates, at
+    cache lengths that put the block inside a chunk, across a span boundary (512) and at the end of a span."""
+    P = synth.DecodeParams(4, 9, 8, 16, 16, seed_prompt=False)
+    eng, W = make(GQAB, P, seed)
+    rng = np.random.default_rng(seed)
+    prompt = synth.prompt(seed, GQAB.vocab, L_prompt, 0.4, 4, 8)
+    eng.reset()
+    eng.prefill(prompt)
+    d = rng.integers(0, GQAB.vocab, P.gamma).tolist()
+    grams = rng.integers(0, GQAB.vocab, (P.K, P.beta)).astype(np.int32)
+    grams[:, 0] = d[-1]
+    eng.phrase_update(grams)
+    pool = oracle_pool(P)
+    for g in grams:
+        pool.insert(g)
+    eng.assemble_candidates(draft=d)
+    tok = eng.block_get()[0]
+    cands = pool.lookup(d[-1], P.K)
+    t2, p2, g2, vis = ob.build_block(len(prompt) - 1, prompt[-1], d, cands)
+    assert tok.tolist() == t2 and len(t2) == P.block_max == 69
+    am, logits = eng.verify_forward(want_logits=True)
+    cache = tf.KVCache(GQAB)
+    ob.prefill(W, cache, list(prompt[:-1]))
+    want = tf.forward(W, cache, t2, p2, vis)
+    got = logits[: len(t2)].cpu().numpy().astype(np.float64)
+    _bf16_tol(got, want)
+    err = np.abs(got - want).max(axis=1)
+    srt = np.sort(want, axis=1)
+    safe = (srt[:, -1] - srt[:, -2]) > 2 * err + 1e-12
+    assert np.array_equal(am[: len(t2)].cpu().numpy()[safe], tf.argmax_rows(want)[safe])
+    eng.close()
