@@ -637,11 +637,7 @@ def test_phrase_level_drafting_edge_cases():
 GQAB = synth.ModelDesc(2, 512, 8, 2, 128, 1024, 1000, 1200, "bf16")   # 4 query heads per kv head, head_dim 128
 
 
-@pytest.mark.parametrize("seed,L_prompt", [(0, 40), (1, 509), (2, 1000), (3, 129)])
-def test_verify_logits_bf16_gqa_head_dim_128(seed, L_prompt):
-    """69 block rows x 4 query heads per kv head = 276 query rows (three rounds of 128) with 8 candidates, at
-    cache lengths that put the block inside a chunk, across a span boundary (512) and at the end of a span."""
-    P = synth.DecodeParams(4, 9, 8, 16, 16, seed_prompt=False)
+def _gqa_case(P, seed, L_prompt):
     eng, W = make(GQAB, P, seed)
     rng = np.random.default_rng(seed)
     prompt = synth.prompt(seed, GQAB.vocab, L_prompt, 0.4, 4, 8)
@@ -658,7 +654,7 @@ def test_verify_logits_bf16_gqa_head_dim_128(seed, L_prompt):
     tok = eng.block_get()[0]
     cands = pool.lookup(d[-1], P.K)
     t2, p2, g2, vis = ob.build_block(len(prompt) - 1, prompt[-1], d, cands)
-    assert tok.tolist() == t2 and len(t2) == P.block_max == 69
+    assert tok.tolist() == t2 and len(t2) == P.block_max
     am, logits = eng.verify_forward(want_logits=True)
     cache = tf.KVCache(GQAB)
     ob.prefill(W, cache, list(prompt[:-1]))
@@ -670,3 +666,16 @@ def test_verify_logits_bf16_gqa_head_dim_128(seed, L_prompt):
     safe = (srt[:, -1] - srt[:, -2]) > 2 * err + 1e-12
     assert np.array_equal(am[: len(t2)].cpu().numpy()[safe], tf.argmax_rows(want)[safe])
     eng.close()
+
+
+@pytest.mark.parametrize("seed,L_prompt", [(0, 40), (1, 509), (2, 1000), (3, 129)])
+def test_verify_logits_bf16_gqa_head_dim_128(seed, L_prompt):
+    """69 block rows x 4 query heads per kv head = 276 query rows (three rounds of 128) with 8 candidates, at
+    cache lengths that put the block inside a chunk, across a span boundary (512) and at the end of a span."""
+    _gqa_case(synth.DecodeParams(4, 9, 8, 16, 16, seed_prompt=False), seed, L_prompt)
+
+
+@pytest.mark.parametrize("gamma,beta,K,L_prompt", [(7, 16, 8, 300), (3, 8, 16, 505)])
+def test_verify_logits_bf16_widest_blocks(gamma, beta, K, L_prompt):
+    """The widest block (128 rows: four rounds of query rows) and the most groups (16 candidates + trunk)."""
+    _gqa_case(synth.DecodeParams(gamma, beta, K, 2, 32, seed_prompt=False), 5, L_prompt)
