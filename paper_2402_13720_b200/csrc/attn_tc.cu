@@ -118,7 +118,9 @@ __global__ void __launch_bounds__(THREADS) attn_span_kernel(const AttnParams p) 
   const uint32_t sm_u = smem_u32(smem);
 
   pdl_trigger();
-  pdl_wait();
+  // Everything up to pdl_wait() reads only what was complete before the forward pass began: the block description
+  // (written by the assembling kernel, which is not launched programmatically and so has finished) and cache rows
+  // below the cache length.  The queries and the block's own K/V rows come from the kernel just before this one.
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int sc = blockIdx.x, kvh = blockIdx.y;
   const int g = p.H / p.Hkv, dkv = p.Hkv * HD;
@@ -181,6 +183,8 @@ __global__ void __launch_bounds__(THREADS) attn_span_kernel(const AttnParams p) 
     if (!__syncthreads_or(any_row)) return;            // nobody in this round reaches the span
     const int n_mt = (min(QR, M_all - m0) + 15) >> 4;  // row tiles that hold query rows; the others are skipped
 
+    stage_common(0, 0);                                 // chunk 0 (its rows below the cache length) is on its way ...
+    pdl_wait();                                         // ... while the previous kernel finishes
     for (int idx = threadIdx.x; idx < QR * CPR; idx += THREADS) {
       int row = idx / CPR, ch = idx % CPR, m = m0 + row;
       uint32_t off = S::OFF_Q + row * ROWB + ((ch ^ (row & 7)) << 4);
@@ -189,7 +193,7 @@ __global__ void __launch_bounds__(THREADS) attn_span_kernel(const AttnParams p) 
       else
         *reinterpret_cast<uint4 *>(smem + off) = make_uint4(0, 0, 0, 0);
     }
-    stage_common(0, 0);                                 // one group: Q and chunk 0
+    cp_commit();                                        // Q is a group of its own, younger than chunk 0
 
     float o[MT][NT2][4], m_run[2 * MT], l_run[2 * MT];
 #pragma unroll
