@@ -606,7 +606,7 @@ def test_phrase_level_drafting_bf16_self_draft():
         res.append(st)
         eng.close()
     assert res[0]["target_calls"] == res[1]["target_calls"] and res[0]["full_accepts"] == res[0]["target_calls"]
-    assert res[1]["draft_calls"] <= res[0]["draft_calls"] == 4 * res[0]["target_calls"]
+    assert res[1]["draft_calls"] < res[0]["draft_calls"] == 4 * res[0]["target_calls"]     # c of Eq. 6 above 1
 
 
 def test_phrase_level_drafting_edge_cases():
