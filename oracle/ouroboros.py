@@ -24,9 +24,10 @@ What the paper fixes and what is this build's reading:
 Pins (tests/test_oracle_ouroboros.py): generated tokens equal plain greedy decoding from the
 definition (Eq. 4) for every seed and flag setting; packed verification equals K separate
 causal forwards (Eq. 8); hand traces under tests/golden/; Eq. 3 / Eq. 9 / Eq. 10 properties;
-compaction equals a fresh prefill.  The pool policy and harvest readings have no counterpart
-in the paper to pin against beyond those traces: PARITY UNPINNED for PhrasePool eviction order
-and harvest_ops window selection.
+compaction equals a fresh prefill.  The pool policy and the harvest readings are this build's
+(the paper is silent); each is fixed by a hand-worked trace: the pool by its policy trace, the matched
+sub-segments and tried phrases by the three step traces, the two extensions (windows of the accepted
+text, windows of the prompt) by trace_harvest_accepted.txt and trace_seed_prompt.txt.
 """
 from __future__ import annotations
 

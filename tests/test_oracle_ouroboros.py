@@ -67,6 +67,39 @@ def test_hand_traces(name):
         assert [list(p) for _, p in pool.export()] == t["pool_after"]
 
 
+def test_hand_trace_harvest_accepted_windows():
+    """Part 3 of harvest_ops (extension): which beta-windows of the text a step's accepted tokens yield."""
+    t = load_trace("trace_harvest_accepted.txt")
+    only = dict(harvest_matched=False, harvest_candidates=False, harvest_accepted=True, seed_prompt=False)
+
+    def windows(seq, n_acc, beta):
+        # block tokens / outputs are irrelevant with the other two parts switched off; A = 0 < gamma
+        ops = ob.harvest_ops([0, 0], [0, 0], 1, beta - 1, 0, 0, seq, n_acc, _params(1, beta, 0, **only))
+        assert all(op[0] == "insert" for op in ops)
+        return [list(op[1]) for op in ops]
+
+    for beta in (3, 4, 5, 6):
+        assert windows(t["text_after"], t["n_accepted"], beta) == t[f"windows_beta{beta}"]
+    assert windows(t["short_text_after"], t["short_n_accepted"], 3) == t["short_windows_beta3"]
+    assert windows(t["single_text_after"], t["single_n_accepted"], 3) == t["single_windows_beta3"]
+    off = dict(only, harvest_accepted=False)
+    assert ob.harvest_ops([0, 0], [0, 0], 1, 2, 0, 0, t["text_after"], 2, _params(1, 3, 0, **off)) == []
+
+
+def test_hand_trace_seed_prompt_windows():
+    """prompt_ops (extension): every beta-window of the prompt, in order; none when the prompt is shorter."""
+    t = load_trace("trace_seed_prompt.txt")
+    for beta in (1, 3, 5, 6):
+        ops = ob.prompt_ops(t["prompt"], beta, _params(2, beta, 1, seed_prompt=True))
+        assert all(op[0] == "insert" for op in ops)
+        assert [list(op[1]) for op in ops] == t[f"windows_beta{beta}"]
+    assert ob.prompt_ops(t["prompt"], 3, _params(2, 3, 1, seed_prompt=False)) == []
+    pool = ob.PhrasePool(1, 4, 3)
+    pool.apply(ob.prompt_ops(t["prompt"], 3, _params(2, 3, 1)))
+    assert [list(p) for _, p in pool.export()] == t["pool_after_beta3"]
+    assert pool.lookup(1, 4) == t["lookup_1"] and pool.lookup(4, 4) == t["lookup_4"]
+
+
 # -------------------------------------------------------------------- mask: packed == separate
 
 @pytest.mark.parametrize("seed", [0, 1])
