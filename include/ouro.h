@@ -166,8 +166,8 @@ int ouro_assemble_causal(ouro_ctx *ctx, int which, const int32_t *tokens_dev, in
 int ouro_block_get(ouro_ctx *ctx, int which, int32_t *tokens_host, int32_t *pos_host, int32_t *group_host,
                    uint64_t *mask_host, int32_t *B);
 
-/* Section 3.2 "a single forward using the attention masking mechanism": runs model `which` on its
- * current block against its KV cache.  Appends the block's K/V at cache slots L..L+B-1, writes the
+/* Section 3.2 / Eq. 8: one forward of model `which` scores every row of its current block (all K
+ * lengthened drafts at once, under the candidate mask) against its KV cache.  Appends the block's K/V at cache slots L..L+B-1, writes the
  * greedy next token of every row to argmax_dev [B] (ties -> smallest id) and, if logits_dev is not
  * NULL, the fp32 logits [B, vocab].  Does not change the cache length.  Asynchronous. */
 int ouro_verify_forward(ouro_ctx *ctx, int which, int32_t *argmax_dev, float *logits_dev);

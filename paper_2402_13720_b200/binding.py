@@ -89,9 +89,10 @@ def lib():
     """The loaded shared library; raises if it has not been built (there is no other implementation)."""
     global _lib
     if _lib is None:
-        if not os.path.exists(_LIB_PATH):
-            raise RuntimeError(f"{_LIB_PATH} is missing: build it with `python -m paper_2402_13720_b200.build`")
-        L = C.CDLL(_LIB_PATH)
+        path = os.environ.get("OURO_LIB") or _LIB_PATH     # OURO_LIB: another build of the same library (trace.py)
+        if not os.path.exists(path):
+            raise RuntimeError(f"{path} is missing: build it with `python -m paper_2402_13720_b200.build`")
+        L = C.CDLL(path)
         for name, (res, args) in _SIGNATURES.items():
             fn = getattr(L, name)
             fn.restype, fn.argtypes = res, args

@@ -31,6 +31,22 @@
 
 #include "ouro_internal.h"
 
+// Optional timeline (compile with -DOURO_TRACE): see gemm_tc.cu.
+#ifdef OURO_TRACE
+__device__ unsigned long long g_attn_trace[512][8];
+__device__ __forceinline__ unsigned long long attn_trace_now() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t)::"memory");
+  return t;
+}
+#define TRACE(slot) do { const int cta_ = blockIdx.y * gridDim.x + blockIdx.x; if (cta_ < 512) g_attn_trace[cta_][slot] = attn_trace_now(); } while (0)
+extern "C" int ouro_trace_read_attn(unsigned long long *out_host) {
+  return (int)cudaMemcpyFromSymbol(out_host, g_attn_trace, sizeof(g_attn_trace));
+}
+#else
+#define TRACE(slot) do { } while (0)
+#endif
+
 namespace {
 
 constexpr int HD = 128;
@@ -194,6 +210,7 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tm_kernel(const __grid_consta
   const int sc = p.n_spans - 1 - blockIdx.x / p.Hkv, kvh = blockIdx.x % p.Hkv, m0 = blockIdx.y * QR;
   const int g = p.H / p.Hkv, dkv = p.Hkv * HD, M_all = g * p.rows, span0 = sc * SPAN;
 
+  if (tid == 0) TRACE(0);
   if (sm_u & 1023) {                                   // the swizzled tiles need a 1024-byte aligned base
     if (tid == 0) atomicExch(p.status, 1);
     return;
@@ -313,7 +330,9 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tm_kernel(const __grid_consta
       ++early;
     }
   }
+  if (tid == 0) TRACE(1);
   pdl_wait();
+  if (tid == 0) TRACE(2);
   // ---- Q tile: K-major, two halves of 64 dims, 128-byte swizzle; rows without a query are zero
   for (int idx = tid; idx < QR * 16; idx += THREADS) {
     const int t = idx >> 4, ch = idx & 15, info = ms->map[t];
@@ -479,6 +498,7 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tm_kernel(const __grid_consta
         const int c0 = span0 + ci * CH;
         const bool active = has && nv > c0 && (go == 63 || go == my_o);
         mbar_wait(&ms->s_ready[b], (i >> 1) & 1, ms, p.status);
+        if (i == 0 && tid == 64) TRACE(3);
         fence_after_sync();
         float alpha = 1.f;
         const int nk = active ? min(nv - c0, CH) : 0;  // keys of this chunk the row sees: tile columns below nk
@@ -578,6 +598,7 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tm_kernel(const __grid_consta
         alpha_prev = alpha;
       }
       if (pending) accumulate(n_items - 1);
+      if (tid == 64) TRACE(4);
       // ---- the span's piece of this row: the two halves of the row sum are added in a fixed order
       float *lsum = reinterpret_cast<float *>(smem + OFF_Q);      // Q is no longer read: every contraction has completed
       lsum[h * QR + t] = l_run;
@@ -603,6 +624,7 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tm_kernel(const __grid_consta
   }
   fence_before_sync();
   __syncthreads();
+  if (tid == 0) TRACE(5);
   if (warp == 1) {
     fence_after_sync();
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(512u));

@@ -22,13 +22,33 @@
 #include <cuda.h>
 
 #include "ouro_internal.h"
+#include "weight_stream.cuh"
 
 void ouro_set_global_error(const std::string &msg);   // api.cu
 
+// Optional timeline of the GEMM launches (compile with -DOURO_TRACE, see paper_2402_13720_b200/trace.py): selected
+// threads of every CTA stamp the global nanosecond timer at fixed points; ouro_trace_read_gemm copies the stamps
+// of the most recent launch of every kind out.  Compiled out by default.
+#ifdef OURO_TRACE
+__device__ unsigned long long g_gemm_trace[8][160][12];
+__device__ __forceinline__ unsigned long long trace_now() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t)::"memory");
+  return t;
+}
+#define TRACE(slot) do { if (blockIdx.x < 160) g_gemm_trace[p.trace_id & 7][blockIdx.x][slot] = trace_now(); } while (0)
+extern "C" int ouro_trace_read_gemm(unsigned long long *out_host) {
+  return (int)cudaMemcpyFromSymbol(out_host, g_gemm_trace, sizeof(g_gemm_trace));
+}
+#else
+#define TRACE(slot) do { } while (0)
+#endif
+
 namespace {
 
-constexpr int TILE_N = 128;       // weight rows per tile (MMA M)
-constexpr int BLOCK_K = 64;       // bf16 elements per k-block: one 128-byte swizzle row
+using ws::BLOCK_K;
+using ws::TILE_N;
+using ws::Span;
 constexpr int A_BYTES = TILE_N * BLOCK_K * 2;
 constexpr int THREADS = 224;      // warp 0 weight TMA, warp 1 MMA, warps 2..5 epilogue, warp 6 activation TMA
 constexpr int MAX_GRID = 160;
@@ -76,6 +96,7 @@ struct GemmParams {
   int *counters;      // [tiles] partial tiles published, zero between launches
   int *done;          // [tiles] contributors that finished their share, zero between launches
   int *status;        // context status word
+  int trace_id;           // which GEMM of the layer this is (timeline builds only)
 };
 
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -152,49 +173,9 @@ __device__ __forceinline__ float ordered_f32(uint32_t u) {
 }
 __device__ __forceinline__ void epi_barrier() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
 
-struct Span {  // one piece of this CTA's work: k-blocks [kb0, kb1) of `tile`
-  int tile, kb0, kb1, n_contrib, slot, first_owner;
-};
-
-// Work of one CTA, identical in every warp role.  The last R = tiles mod grid tiles are cut stream-K
-// fashion into equal contiguous spans of the (tile, k-block) space and come first, so that their partial
-// sums are added up while the whole tiles (tile c, c + grid, ...) that follow are still streaming.
-struct SpanWalker {
-  int kb, per, t0, it, end, whole;
-  __device__ SpanWalker(const GemmParams &p) {
-    kb = p.kb;
-    t0 = (p.tiles / (int)gridDim.x) * (int)gridDim.x;      // tiles [0, t0) are handled whole
-    int total = (p.tiles - t0) * kb;
-    per = (total + gridDim.x - 1) / gridDim.x;
-    it = min(total, (int)blockIdx.x * per);
-    end = min(total, it + per);
-    whole = blockIdx.x;
-  }
-  __device__ int owner_slot(int tile, int owner) const { return ((tile - t0) * kb <= owner * per) ? 0 : 1; }
-  __device__ bool next(Span &s) {
-    if (it < end) {
-      int rel = it / kb;
-      s.tile = t0 + rel;
-      s.kb0 = it - rel * kb;
-      s.kb1 = min(kb, s.kb0 + (end - it));
-      s.first_owner = (rel * kb) / per;
-      s.n_contrib = (rel * kb + kb - 1) / per - s.first_owner + 1;
-      s.slot = owner_slot(s.tile, blockIdx.x);               // first or last piece of this CTA
-      it += s.kb1 - s.kb0;
-      return true;
-    }
-    if (whole < t0) {
-      s.tile = whole;
-      s.kb0 = 0;
-      s.kb1 = kb;
-      s.n_contrib = 1;
-      s.slot = 0;
-      s.first_owner = blockIdx.x;
-      whole += gridDim.x;
-      return true;
-    }
-    return false;
-  }
+// The schedule of this launch for CTA blockIdx.x (see weight_stream.cuh).
+struct SpanWalker : ws::SpanWalker {
+  __device__ SpanWalker(const GemmParams &p) : ws::SpanWalker(p.tiles, p.kb, (int)gridDim.x, (int)blockIdx.x) {}
 };
 
 // Locates a tile: which stacked matrix, its first row there, and the first output column.
@@ -241,6 +222,7 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_tc_kernel(const __grid_consta
   int *spos = (int *)(rs + OURO_MAX_ROWS);                  // [128] token positions (rotary table rows), QKV epilogue
 
   pdl_trigger();
+  if (threadIdx.x == 0) TRACE(0);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int acc_cols = p.t_pad <= 32 ? 32 : p.t_pad <= 64 ? 64 : 128;   // columns per accumulator buffer
 
@@ -295,12 +277,14 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_tc_kernel(const __grid_consta
           issue(s, kb, st);
         }
       }
+      TRACE(8);
       if (!ok) { *abort_flag = 1; atomicExch(p.status, 1); }
     }
   } else if (warp == 6) {
     // ---------------------------------------------------------------- activation producer
     if (lane == 0) {
       pdl_wait();                                  // the activations are the previous kernel's output
+      TRACE(1);
       SpanWalker w(p);
       Span s;
       uint32_t n = 0;
@@ -334,6 +318,7 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_tc_kernel(const __grid_consta
           int st = n % p.stages;
           ok = mbar_wait(&full[st], (n / p.stages) & 1) && !*abort_flag;
           if (!ok) break;
+          if (n == 0) TRACE(2);
           fence_after_sync();
           uint32_t sa = smem_u32(ring + (size_t)st * stage_bytes), sb = sa + A_BYTES;
           uint64_t da = smem_desc_sw128(sa), db = smem_desc_sw128(sb);
@@ -345,6 +330,7 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_tc_kernel(const __grid_consta
         mma_commit(&acc_full[a]);
         ++item;
       }
+      TRACE(3);
       if (!ok) { *abort_flag = 1; atomicExch(p.status, 1); }
     }
   } else {
@@ -380,6 +366,7 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_tc_kernel(const __grid_consta
         ok = wait_flag[0] != 0;
         epi_barrier();
         if (!ok) break;
+        if (et == 0) TRACE(6);                     // the partial tiles of the other contributors are there
         __threadfence();
         if (p.mode == MODE_SWIGLU) {
           const int F = p.a_rows[0];
@@ -613,6 +600,7 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_tc_kernel(const __grid_consta
       epi_barrier();
       ok = wait_flag[a] != 0;
       if (!ok) break;
+      if (et == 0) TRACE(4);                       // overwritten per item: the last accumulator's arrival remains
       fence_after_sync();
       const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + a * acc_cols;
       int seg = 0, row0 = 0, col0 = 0, valid = TILE_N;
@@ -761,7 +749,9 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_tc_kernel(const __grid_consta
       }
       ++item;
     }
+    if (et == 0) TRACE(5);
     run_fixups();
+    if (et == 0) TRACE(7);
     if (!ok && et == 0) { *abort_flag = 1; atomicExch(p.status, 1); }
   }
   // ------------------------------------------------------------------ teardown
@@ -917,6 +907,61 @@ void ouro_fast_teardown(ouro_ctx *c) {
   c->fast = nullptr;
 }
 
+// The weight side of one GEMM of the forward: which matrices, how they are tiled, how long K is.
+enum { G_QKV = 0, G_WO = 1, G_GATEUP = 2, G_DOWN = 3, G_HEAD = 4 };
+struct WeightSide {
+  CUtensorMap a[3];
+  int a_tiles[3] = {0, 0, 0}, a_rows[3] = {0, 0, 0}, a_count = 1, tiles = 0, K = 0;
+  bool swiglu = false;
+};
+static WeightSide weight_side(const ouro_model_desc &d, const FastModel &fm, int l, int kind) {
+  auto tiles = [](int n) { return (n + TILE_N - 1) / TILE_N; };
+  const int dq = d.n_heads * d.head_dim, dkv = d.n_kv_heads * d.head_dim;
+  WeightSide w;
+  switch (kind) {
+    case G_QKV: {
+      const LayerMaps &lm = fm.layers[l];
+      w.a[0] = lm.wq; w.a[1] = lm.wk; w.a[2] = lm.wv;
+      w.a_tiles[0] = tiles(dq); w.a_tiles[1] = tiles(dkv); w.a_tiles[2] = tiles(dkv);
+      w.a_rows[0] = dq; w.a_rows[1] = dkv; w.a_rows[2] = dkv;
+      w.a_count = 3;
+      w.tiles = w.a_tiles[0] + w.a_tiles[1] + w.a_tiles[2];
+      w.K = d.d_model;
+      break;
+    }
+    case G_WO:
+      w.a[0] = fm.layers[l].wo; w.a_tiles[0] = tiles(d.d_model); w.a_rows[0] = d.d_model;
+      w.tiles = w.a_tiles[0];
+      w.K = dq;
+      break;
+    case G_GATEUP:
+      w.a[0] = fm.layers[l].wg; w.a[1] = fm.layers[l].wu; w.a_rows[0] = d.d_ffn; w.a_count = 2;
+      w.tiles = (d.d_ffn + 63) / 64;
+      w.K = d.d_model;
+      w.swiglu = true;
+      break;
+    case G_DOWN:
+      w.a[0] = fm.layers[l].wd; w.a_tiles[0] = tiles(d.d_model); w.a_rows[0] = d.d_model;
+      w.tiles = w.a_tiles[0];
+      w.K = d.d_ffn;
+      break;
+    default:
+      w.a[0] = fm.head; w.a_tiles[0] = tiles(d.vocab); w.a_rows[0] = d.vocab;
+      w.tiles = w.a_tiles[0];
+      w.K = d.d_model;
+      break;
+  }
+  return w;
+}
+static void set_weights(GemmParams &p, const WeightSide &w) {
+  for (int i = 0; i < 3; ++i) { p.a[i] = w.a[i]; p.a_tiles[i] = w.a_tiles[i]; p.a_rows[i] = w.a_rows[i]; }
+  p.a_count = w.a_count;
+  p.tiles = w.tiles;
+}
+static int grid_for(const FastState &s, int tiles, int kb) {
+  const long total = (long)tiles * kb;
+  return total < s.grid ? (int)total : s.grid;
+}
 static void launch_gemm_tc(ouro_ctx *c, GemmParams &p, const CUtensorMap *xmaps, int K, int rows) {
   OURO_COUNT_LAUNCH();
   FastState &s = c->fast->s;
@@ -929,9 +974,7 @@ static void launch_gemm_tc(ouro_ctx *c, GemmParams &p, const CUtensorMap *xmaps,
   p.counters = s.counters;
   p.done = s.counters + MAX_TILES;
   p.status = &c->st->status;
-  int total = p.tiles * p.kb;
-  int grid = total < s.grid ? total : s.grid;
-  launch_pdl(gemm_tc_kernel, grid, THREADS, (size_t)s.smem_max, c->stream, p);
+  launch_pdl(gemm_tc_kernel, grid_for(s, p.tiles, p.kb), THREADS, (size_t)s.smem_max, c->stream, p);
 }
 
 // Embedding rows into the residual stream, plus what the first norm's consumer needs: bf16(gain * x) and each
@@ -982,7 +1025,6 @@ int ouro_fast_layer(ouro_ctx *c, int which, int l, int rows) {
   const int dq = d.n_heads * d.head_dim, dkv = d.n_kv_heads * d.head_dim;
   Activations &a = c->a;
   cudaStream_t s = c->stream;
-  LayerMaps &lm = fm.layers[l];
   auto tiles = [](int n) { return (n + TILE_N - 1) / TILE_N; };
   // a.xn holds bf16(attn_norm * x) and ss the sums of squares, left by the embedding or the previous layer's down GEMM
   float *ss = c->fast->s.ss;
@@ -992,11 +1034,8 @@ int ouro_fast_layer(ouro_ctx *c, int which, int l, int rows) {
   {
     ProfScope ps(c, OURO_PROF_QKV);
     GemmParams p{};
-    p.a[0] = lm.wq; p.a[1] = lm.wk; p.a[2] = lm.wv;
-    p.a_tiles[0] = tiles(dq); p.a_tiles[1] = tiles(dkv); p.a_tiles[2] = tiles(dkv);
-    p.a_rows[0] = dq; p.a_rows[1] = dkv; p.a_rows[2] = dkv;
-    p.a_count = 3;
-    p.tiles = p.a_tiles[0] + p.a_tiles[1] + p.a_tiles[2];
+    set_weights(p, weight_side(d, fm, l, G_QKV));
+    p.trace_id = G_QKV;
     consume(p);
     const bool fused_rope = d.head_dim == 64 || d.head_dim == 128;   // tiles then hold whole heads
     if (fused_rope) {
@@ -1032,9 +1071,9 @@ int ouro_fast_layer(ouro_ctx *c, int which, int l, int rows) {
   {
     ProfScope ps(c, OURO_PROF_WO);
     GemmParams p{};
-    p.a[0] = lm.wo; p.a_tiles[0] = tiles(d.d_model); p.a_rows[0] = d.d_model; p.a_count = 1;
+    set_weights(p, weight_side(d, fm, l, G_WO));
+    p.trace_id = G_WO;
     p.mode = MODE_RESIDUAL;
-    p.tiles = p.a_tiles[0];
     p.out_f32 = a.x;
     p.ldo = d.d_model;
     produce(p, M.ffn_norm[l]);
@@ -1043,9 +1082,9 @@ int ouro_fast_layer(ouro_ctx *c, int which, int l, int rows) {
   {
     ProfScope ps(c, OURO_PROF_GATEUP);
     GemmParams p{};
-    p.a[0] = lm.wg; p.a[1] = lm.wu; p.a_rows[0] = d.d_ffn; p.a_count = 2;
+    set_weights(p, weight_side(d, fm, l, G_GATEUP));
+    p.trace_id = G_GATEUP;
     p.mode = MODE_SWIGLU;
-    p.tiles = (d.d_ffn + 63) / 64;
     p.out_bf16 = (__nv_bfloat16 *)a.act;
     consume(p);
     launch_gemm_tc(c, p, fm.x_d, d.d_model, rows);
@@ -1053,9 +1092,9 @@ int ouro_fast_layer(ouro_ctx *c, int which, int l, int rows) {
   {
     ProfScope ps(c, OURO_PROF_DOWN);
     GemmParams p{};
-    p.a[0] = lm.wd; p.a_tiles[0] = tiles(d.d_model); p.a_rows[0] = d.d_model; p.a_count = 1;
+    set_weights(p, weight_side(d, fm, l, G_DOWN));
+    p.trace_id = G_DOWN;
     p.mode = MODE_RESIDUAL;
-    p.tiles = p.a_tiles[0];
     p.out_f32 = a.x;
     p.ldo = d.d_model;
     produce(p, l + 1 < d.n_layers ? M.attn_norm[l + 1] : M.final_norm);
@@ -1107,9 +1146,9 @@ int ouro_fast_head(ouro_ctx *c, int which, int rows, float *logits, int32_t *arg
   {
     ProfScope ps(c, OURO_PROF_HEAD);
     GemmParams p{};
-    p.a[0] = fm.head; p.a_tiles[0] = (d.vocab + TILE_N - 1) / TILE_N; p.a_rows[0] = d.vocab; p.a_count = 1;
+    set_weights(p, weight_side(d, fm, 0, G_HEAD));
+    p.trace_id = G_HEAD;
     p.mode = MODE_HEAD;
-    p.tiles = p.a_tiles[0];
     p.out_f32 = logits;
     p.ldo = d.vocab;
     p.tile_max = c->fast->s.tile_max;
