@@ -172,6 +172,9 @@ __device__ __forceinline__ float ordered_f32(uint32_t u) {
   return __uint_as_float((u & 0x80000000u) ? (u & 0x7fffffffu) : ~u);
 }
 __device__ __forceinline__ void epi_barrier() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
+// one half (64 threads) of the epilogue warps; grp = 0 or 1
+__device__ __forceinline__ void group_barrier(int grp) { asm volatile("bar.sync %0, 64;" ::"r"(2 + grp) : "memory"); }
+constexpr int STAGE_TOK = 64;     // tokens of a whole tile parked in shared memory at a time (64 x 128 fp32 = 32 KB)
 
 // The schedule of this launch for CTA blockIdx.x (see weight_stream.cuh).
 struct SpanWalker : ws::SpanWalker {
@@ -193,31 +196,18 @@ __device__ __forceinline__ void locate(const GemmParams &p, int tile, int &seg, 
   valid = min(TILE_N, p.a_rows[seg] - row0);
 }
 
-// Final values of one output row n (this thread) for tokens t0..t0+15.
-__device__ __forceinline__ void store_chunk(const GemmParams &p, int col, bool n_ok, int t0, const float *v) {
-  if (!n_ok || !p.out_f32) return;
-#pragma unroll
-  for (int i = 0; i < 16; ++i) {
-    int t = t0 + i;
-    if (t < p.rows) {
-      float *y = p.out_f32 + (size_t)t * p.ldo + col;
-      *y = p.mode == MODE_RESIDUAL ? *y + v[i] : v[i];
-    }
-  }
-}
-
 __global__ void __launch_bounds__(THREADS, 1) gemm_tc_kernel(const __grid_constant__ GemmParams p) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t *smem = (uint8_t *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
   const int b_bytes = p.t_pad * BLOCK_K * 2;
   const int stage_bytes = A_BYTES + b_bytes;
   uint8_t *ring = smem;
-  float *xchg = (float *)(ring + (size_t)p.stages * stage_bytes);          // [64][t_pad] up values (SwiGLU)
+  float *xchg = (float *)(ring + (size_t)p.stages * stage_bytes);          // [64 tokens][128] accumulators of a whole tile
   uint64_t *bars = (uint64_t *)((uint8_t *)xchg + 64 * OURO_MAX_ROWS * 4);
   uint64_t *full = bars, *empty = bars + 16, *acc_full = bars + 32, *acc_empty = bars + 34;
   uint32_t *tmem_base_p = (uint32_t *)(bars + 36);
   volatile int *abort_flag = (volatile int *)(bars + 37);
-  volatile int *wait_flag = (volatile int *)(bars + 39);   // [2]: outcome of the epilogue's accumulator wait
+  volatile int *wait_flag = (volatile int *)(bars + 39);   // [0..1]: outcome of an accumulator wait; [2]: a fix-up gave up; [4..5]: outcome of a fix-up group's wait
   float *rs = (float *)(bars + 48);                         // [128] per-token factor 1/rms of the consumed activations
   int *spos = (int *)(rs + OURO_MAX_ROWS);                  // [128] token positions (rotary table rows), QKV epilogue
 
@@ -345,235 +335,297 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_tc_kernel(const __grid_consta
     bool ok = true;
     float v[16];
     int pend_tile[2], pend_n[2], pend_first[2], n_pend = 0;     // partial tiles this CTA contributed to (<= 2)
+    float *stage = xchg;                                         // [STAGE_TOK tokens][128 tile rows] fp32
 
-    // Partial tiles: every contributor of a tile adds up a share of its tokens (token t belongs to contributor
-    // t mod n), in ascending K order.  Called once this CTA has published all its own partials, so waiting for
-    // the others cannot form a cycle; the wait is bounded all the same.  Loads of a batch of four tokens and four
-    // contributors are issued together, so a pass costs about one L2 round trip.
-    auto run_fixups = [&]() {
-      for (int k = 0; ok && k < n_pend; ++k) {
-        const int tile = pend_tile[k], n = pend_n[k], first = pend_first[k], my = (int)blockIdx.x - first;
-        if (et == 0) {
-          int seen = 0;
-          for (uint32_t i = 0; i < (1u << 22); ++i) {
-            asm volatile("ld.acquire.gpu.global.b32 %0, [%1];" : "=r"(seen) : "l"(p.counters + tile) : "memory");
-            if (seen >= n) break;
-            __nanosleep(20);
-          }
-          wait_flag[0] = seen >= n && !*abort_flag;
+    // Finishing tokens of a tile.  Whatever produced the accumulator values - this CTA's own whole tile, parked
+    // in shared memory token-major, or the partial tiles of all contributors in scratch - the last step is the
+    // same: a group of G threads walks over "its" tokens, a warp's 32 lanes holding the tile's 128 rows (= output
+    // columns) four apiece, so every global access is a 16-byte piece of a contiguous 512-byte row.
+    //   whole tile:  stg != NULL; tokens t_base + tg + TG j below t_lim (one staged chunk of tokens)
+    //   split tile:  stg == NULL; tokens my + n (tg + TG j): contributor `my` of n takes the tokens t = my (mod n)
+    //                and adds the partials up in ascending K order; it first waits (bounded) until all n have
+    //                published, and fetches what the epilogue itself reads (residual stream, rotary table) for its
+    //                first tokens before that wait.
+    // Returns false when the wait gave up.
+    auto others_there = [&](int tile, int n, int gi, int grp, int G) -> bool {
+      if (gi == 0) {
+        int seen = 0;
+        for (uint32_t i = 0; i < (1u << 22); ++i) {
+          asm volatile("ld.acquire.gpu.global.b32 %0, [%1];" : "=r"(seen) : "l"(p.counters + tile) : "memory");
+          if (seen >= n) break;
         }
-        epi_barrier();
-        ok = wait_flag[0] != 0;
-        epi_barrier();
-        if (!ok) break;
-        if (et == 0) TRACE(6);                     // the partial tiles of the other contributors are there
-        __threadfence();
-        if (p.mode == MODE_SWIGLU) {
-          const int F = p.a_rows[0];
-          const int ng = et & 15, tg = et >> 4;                       // 4 features; tokens my + n*(tg + 8j)
-          const int feat = tile * 64 + 4 * ng;
-          for (int tb = my + n * tg; tb < p.rows; tb += n * 32) {
-            float4 g[4], u[4];
+        wait_flag[4 + grp] = seen >= n && !*abort_flag;
+        TRACE(6);
+      }
+      if (G == 128) epi_barrier(); else group_barrier(grp);
+      __threadfence();
+      if (gi == 0 && grp == 0) TRACE(9);
+      return wait_flag[4 + grp] != 0;
+    };
+
+    auto finish_plain = [&](int tile, int gi, int G, int grp, int my, int n, int first, const float *stg, int t_base,
+                            int t_lim) -> bool {
+      int seg, row0, col0, valid;
+      locate(p, tile, seg, row0, col0, valid);
+      const int ng = gi & 31, tg = gi >> 5, TG = G >> 5;
+      const int col = col0 + 4 * ng;
+      const bool full4 = 4 * ng + 3 < valid;
+      const int js = n * TG;                                         // token step inside a batch of four
+      const int cm = row0 + 4 * ng;                                  // first of this thread's 4 columns inside q, k or v
+      const int half = p.head_dim >> 1;
+      const bool upper = (cm & half) != 0;
+      const bool res_norm = p.mode == MODE_RESIDUAL && p.gain != nullptr;
+      const bool rope = p.mode == MODE_QKV && seg != 2;
+      float gn[4] = {0.f, 0.f, 0.f, 0.f};
+      if (res_norm) {
 #pragma unroll
-            for (int j = 0; j < 4; ++j) g[j] = u[j] = make_float4(0.f, 0.f, 0.f, 0.f);
-            for (int c0 = 0; c0 < n; c0 += 4) {
-              float4 tg4[4][4], tu4[4][4];
+        for (int e = 0; e < 4; ++e) gn[e] = 4 * ng + e < valid ? __bfloat162float(p.gain[col + e]) : 0.f;
+      }
+      // what the epilogue reads besides the accumulators, for the four tokens of a batch at once
+      auto load_ops = [&](int tb, float4 *oa, float4 *ob) {
 #pragma unroll
-              for (int cc = 0; cc < 4; ++cc) {
-                const int owner = first + c0 + cc;
-                const float *src = p.scratch + ((size_t)owner * 2 + w.owner_slot(tile, owner)) * SLOT_FLOATS + 4 * ng;
+        for (int j = 0; j < 4; ++j) {
+          const int t = tb + j * js;
+          oa[j] = ob[j] = make_float4(0.f, 0.f, 0.f, 0.f);
+          if (t >= t_lim) continue;
+          if (res_norm) {
+            const float *y = p.out_f32 + (size_t)t * p.ldo + col;
+            if (full4) {
+              oa[j] = *reinterpret_cast<const float4 *>(y);
+            } else {
+              if (4 * ng < valid) oa[j].x = y[0];
+              if (4 * ng + 1 < valid) oa[j].y = y[1];
+              if (4 * ng + 2 < valid) oa[j].z = y[2];
+            }
+          } else if (rope) {
+            const size_t ti = (size_t)spos[t] * half + (cm & (half - 1));
+            oa[j] = *reinterpret_cast<const float4 *>(p.cos_t + ti);
+            ob[j] = *reinterpret_cast<const float4 *>(p.sin_t + ti);
+          }
+        }
+      };
+      const int tb0 = t_base + my + n * tg;
+      float4 oa[4], ob[4];
+      if (tb0 < t_lim) load_ops(tb0, oa, ob);
+      if (!stg && !others_there(tile, n, gi, grp, G)) return false;
+      for (int tb = tb0; tb < t_lim; tb += 4 * js) {                 // tokens are uniform inside a warp
+        if (tb != tb0) load_ops(tb, oa, ob);
+        float4 acc[4];
+        if (stg) {
 #pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                  const int t = tb + j * n * 8;
-                  const bool in = c0 + cc < n && t < p.rows;
-                  tg4[cc][j] = in ? __ldcg((const float4 *)(src + (size_t)t * TILE_N)) : make_float4(0.f, 0.f, 0.f, 0.f);
-                  tu4[cc][j] = in ? __ldcg((const float4 *)(src + (size_t)t * TILE_N + 64)) : make_float4(0.f, 0.f, 0.f, 0.f);
-                }
+          for (int j = 0; j < 4; ++j) {
+            const int t = tb + j * js;
+            acc[j] = t < t_lim ? *reinterpret_cast<const float4 *>(stg + (size_t)(t - t_base) * TILE_N + 4 * ng)
+                               : make_float4(0.f, 0.f, 0.f, 0.f);
+          }
+        } else {
+#pragma unroll
+          for (int j = 0; j < 4; ++j) acc[j] = make_float4(0.f, 0.f, 0.f, 0.f);
+          for (int c0 = 0; c0 < n; c0 += 4) {
+            float4 tmp[4][4];
+#pragma unroll
+            for (int cc = 0; cc < 4; ++cc) {
+              const int owner = first + c0 + cc;
+              const float *src = p.scratch + ((size_t)owner * 2 + w.owner_slot(tile, owner)) * SLOT_FLOATS + 4 * ng;
+#pragma unroll
+              for (int j = 0; j < 4; ++j) {
+                const int t = tb + j * js;
+                tmp[cc][j] = (c0 + cc < n && t < t_lim) ? __ldcg((const float4 *)(src + (size_t)t * TILE_N))
+                                                         : make_float4(0.f, 0.f, 0.f, 0.f);
               }
+            }
 #pragma unroll
-              for (int cc = 0; cc < 4; ++cc)
+            for (int cc = 0; cc < 4; ++cc)
 #pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                  g[j].x += tg4[cc][j].x; g[j].y += tg4[cc][j].y; g[j].z += tg4[cc][j].z; g[j].w += tg4[cc][j].w;
-                  u[j].x += tu4[cc][j].x; u[j].y += tu4[cc][j].y; u[j].z += tu4[cc][j].z; u[j].w += tu4[cc][j].w;
+              for (int j = 0; j < 4; ++j) {
+                acc[j].x += tmp[cc][j].x; acc[j].y += tmp[cc][j].y; acc[j].z += tmp[cc][j].z; acc[j].w += tmp[cc][j].w;
+              }
+          }
+        }
+        if (res_norm) {
+          // new residual stream, its bf16(gain * x) image for the next GEMM, and this tile's sums of squares
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            const int t = tb + j * js;
+            if (t >= t_lim) continue;                                // uniform inside the warp
+            float *y = p.out_f32 + (size_t)t * p.ldo + col;
+            const float yn[4] = {oa[j].x + acc[j].x, oa[j].y + acc[j].y, oa[j].z + acc[j].z, oa[j].w + acc[j].w};
+            float sq = 0.f;
+#pragma unroll
+            for (int e = 0; e < 4; ++e)
+              if (4 * ng + e < valid) sq += yn[e] * yn[e];
+            if (full4) {
+              *reinterpret_cast<float4 *>(y) = make_float4(yn[0], yn[1], yn[2], yn[3]);
+              __nv_bfloat162 lo = __floats2bfloat162_rn(gn[0] * yn[0], gn[1] * yn[1]);
+              __nv_bfloat162 hi = __floats2bfloat162_rn(gn[2] * yn[2], gn[3] * yn[3]);
+              *reinterpret_cast<uint2 *>(p.xb + (size_t)t * p.ldo + col) = make_uint2(*(uint32_t *)&lo, *(uint32_t *)&hi);
+            } else {
+#pragma unroll
+              for (int e = 0; e < 4; ++e)
+                if (4 * ng + e < valid) {
+                  y[e] = yn[e];
+                  p.xb[(size_t)t * p.ldo + col + e] = __float2bfloat16_rn(gn[e] * yn[e]);
                 }
             }
 #pragma unroll
-            for (int j = 0; j < 4; ++j) {
-              const int t = tb + j * n * 8;
-              if (t < p.rows) {
-                const float r = rs[t];
-                g[j].x *= r; g[j].y *= r; g[j].z *= r; g[j].w *= r;
-                u[j].x *= r; u[j].y *= r; u[j].z *= r; u[j].w *= r;
-              }
-              if (t < p.rows && feat < F) {
-                __nv_bfloat162 lo = __floats2bfloat162_rn(g[j].x / (1.0f + __expf(-g[j].x)) * u[j].x, g[j].y / (1.0f + __expf(-g[j].y)) * u[j].y);
-                __nv_bfloat162 hi = __floats2bfloat162_rn(g[j].z / (1.0f + __expf(-g[j].z)) * u[j].z, g[j].w / (1.0f + __expf(-g[j].w)) * u[j].w);
-                *(uint2 *)(p.out_bf16 + (size_t)t * F + feat) = make_uint2(*(uint32_t *)&lo, *(uint32_t *)&hi);
-              }
+            for (int o = 16; o; o >>= 1) sq += __shfl_xor_sync(0xffffffffu, sq, o);
+            if (lane == 0) p.ss_out[(size_t)tile * OURO_MAX_ROWS + t] = sq;
+          }
+          continue;
+        }
+        if (p.mode == MODE_QKV) {
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            const int t = tb + j * js;
+            if (t >= t_lim) continue;                                // uniform inside the warp
+            const float r = rs[t];
+            const float vals[4] = {acc[j].x * r, acc[j].y * r, acc[j].z * r, acc[j].w * r};
+            float other[4];
+#pragma unroll
+            for (int e = 0; e < 4; ++e) other[e] = __shfl_xor_sync(0xffffffffu, vals[e], half >> 2);
+            const float cs[4] = {oa[j].x, oa[j].y, oa[j].z, oa[j].w}, sn[4] = {ob[j].x, ob[j].y, ob[j].z, ob[j].w};
+            float rv[4];
+#pragma unroll
+            for (int e = 0; e < 4; ++e)
+              rv[e] = seg == 2 ? vals[e] : (upper ? vals[e] * cs[e] + other[e] * sn[e] : vals[e] * cs[e] - other[e] * sn[e]);
+            __nv_bfloat16 *dst = seg == 0 ? p.q_out + (size_t)t * p.dq + cm
+                               : seg == 1 ? p.k_out + (size_t)(p.L + t) * p.dkv + cm
+                                          : p.v_out + (size_t)(p.L + t) * p.dkv + cm;
+            if (full4) {
+              __nv_bfloat162 lo = __floats2bfloat162_rn(rv[0], rv[1]), hi = __floats2bfloat162_rn(rv[2], rv[3]);
+              *reinterpret_cast<uint2 *>(dst) = make_uint2(*(uint32_t *)&lo, *(uint32_t *)&hi);
+            } else {
+#pragma unroll
+              for (int e = 0; e < 4; ++e)
+                if (4 * ng + e < valid) dst[e] = __float2bfloat16_rn(rv[e]);
+            }
+          }
+          continue;
+        }
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          const int t = tb + j * js;
+          if (t >= t_lim) continue;                                  // uniform inside the warp
+          const float r = rs[t];
+          const float vals[4] = {acc[j].x * r, acc[j].y * r, acc[j].z * r, acc[j].w * r};
+          if (p.mode == MODE_HEAD) {                                 // the warp's 32 lanes hold the tile's 128 columns
+            uint32_t bu = 0;
+            int bi = col;
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+              uint32_t uo = ordered_u32(vals[e]);
+              if (4 * ng + e < valid && uo > bu) { bu = uo; bi = col + e; }
+            }
+            const uint32_t mx = __reduce_max_sync(0xffffffffu, bu);
+            const int src_lane = __ffs(__ballot_sync(0xffffffffu, bu == mx)) - 1;   // lowest lane = smallest index
+            bi = __shfl_sync(0xffffffffu, bi, src_lane);
+            if (lane == 0) {
+              p.tile_max[(size_t)tile * OURO_MAX_ROWS + t] = ordered_f32(mx);
+              p.tile_arg[(size_t)tile * OURO_MAX_ROWS + t] = bi;
+            }
+          }
+          if (p.out_f32) {
+            float *y = p.out_f32 + (size_t)t * p.ldo + col;
+            const bool add = p.mode == MODE_RESIDUAL;
+            if (full4 && ((p.ldo & 3) == 0)) {
+              float4 o4 = make_float4(vals[0], vals[1], vals[2], vals[3]);
+              if (add) { const float4 y4 = *reinterpret_cast<const float4 *>(y); o4.x += y4.x; o4.y += y4.y; o4.z += y4.z; o4.w += y4.w; }
+              *reinterpret_cast<float4 *>(y) = o4;
+            } else {
+#pragma unroll
+              for (int e = 0; e < 4; ++e)
+                if (4 * ng + e < valid) y[e] = add ? y[e] + vals[e] : vals[e];
+            }
+          }
+        }
+      }
+      return true;
+    };
+
+    // SiLU(gate) * up: a tile holds 64 output features, gate in tile rows 0..63 and up in rows 64..127
+    auto finish_swiglu = [&](int tile, int gi, int G, int grp, int my, int n, int first, const float *stg, int t_base,
+                             int t_lim) -> bool {
+      const int F = p.a_rows[0];
+      const int ng = gi & 15, tg = gi >> 4, TG = G >> 4;             // 4 features; tokens my + n (tg + TG j)
+      const int feat = tile * 64 + 4 * ng;
+      const int js = n * TG;
+      if (!stg && !others_there(tile, n, gi, grp, G)) return false;
+      for (int tb = t_base + my + n * tg; tb < t_lim; tb += 4 * js) {
+        float4 g[4], u[4];
+        if (stg) {
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            const int t = tb + j * js;
+            g[j] = u[j] = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (t < t_lim) {
+              g[j] = *reinterpret_cast<const float4 *>(stg + (size_t)(t - t_base) * TILE_N + 4 * ng);
+              u[j] = *reinterpret_cast<const float4 *>(stg + (size_t)(t - t_base) * TILE_N + 64 + 4 * ng);
             }
           }
         } else {
-          int seg, row0, col0, valid;
-          locate(p, tile, seg, row0, col0, valid);
-          const int ng = et & 31, tg = et >> 5;                       // 4 columns; tokens my + n*(tg + 4j)
-          const int col = col0 + 4 * ng;
-          for (int tb = my + n * tg; tb < p.rows; tb += n * 16) {     // tokens are uniform inside a warp
-            float4 acc[4];
 #pragma unroll
-            for (int j = 0; j < 4; ++j) acc[j] = make_float4(0.f, 0.f, 0.f, 0.f);
-            for (int c0 = 0; c0 < n; c0 += 4) {
-              float4 tmp[4][4];
+          for (int j = 0; j < 4; ++j) g[j] = u[j] = make_float4(0.f, 0.f, 0.f, 0.f);
+          for (int c0 = 0; c0 < n; c0 += 4) {
+            float4 tg4[4][4], tu4[4][4];
 #pragma unroll
-              for (int cc = 0; cc < 4; ++cc) {
-                const int owner = first + c0 + cc;
-                const float *src = p.scratch + ((size_t)owner * 2 + w.owner_slot(tile, owner)) * SLOT_FLOATS + 4 * ng;
-#pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                  const int t = tb + j * n * 4;
-                  tmp[cc][j] = (c0 + cc < n && t < p.rows) ? __ldcg((const float4 *)(src + (size_t)t * TILE_N))
-                                                           : make_float4(0.f, 0.f, 0.f, 0.f);
-                }
-              }
-#pragma unroll
-              for (int cc = 0; cc < 4; ++cc)
-#pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                  acc[j].x += tmp[cc][j].x; acc[j].y += tmp[cc][j].y; acc[j].z += tmp[cc][j].z; acc[j].w += tmp[cc][j].w;
-                }
-            }
-            // What the epilogue reads (residual stream, rotary table) is fetched for the four tokens at once,
-            // ahead of the arithmetic and the stores: one round trip to L2 per pass instead of one per token.
-            const bool full4 = 4 * ng + 3 < valid;
-            if (p.mode == MODE_RESIDUAL && p.gain) {
-              float4 yv[4];
+            for (int cc = 0; cc < 4; ++cc) {
+              const int owner = first + c0 + cc;
+              const float *src = p.scratch + ((size_t)owner * 2 + w.owner_slot(tile, owner)) * SLOT_FLOATS + 4 * ng;
 #pragma unroll
               for (int j = 0; j < 4; ++j) {
-                const int t = tb + j * n * 4;
-                yv[j] = make_float4(0.f, 0.f, 0.f, 0.f);
-                if (t < p.rows) {
-                  const float *y = p.out_f32 + (size_t)t * p.ldo + col;
-                  if (full4) {
-                    yv[j] = *reinterpret_cast<const float4 *>(y);
-                  } else {
-                    if (4 * ng < valid) yv[j].x = y[0];
-                    if (4 * ng + 1 < valid) yv[j].y = y[1];
-                    if (4 * ng + 2 < valid) yv[j].z = y[2];
-                  }
-                }
-              }
-              float gn[4];
-#pragma unroll
-              for (int e = 0; e < 4; ++e) gn[e] = 4 * ng + e < valid ? __bfloat162float(p.gain[col + e]) : 0.f;
-#pragma unroll
-              for (int j = 0; j < 4; ++j) {
-                const int t = tb + j * n * 4;
-                if (t >= p.rows) continue;                            // uniform inside the warp
-                float *y = p.out_f32 + (size_t)t * p.ldo + col;
-                const float yn[4] = {yv[j].x + acc[j].x, yv[j].y + acc[j].y, yv[j].z + acc[j].z, yv[j].w + acc[j].w};
-                float sq = 0.f;
-#pragma unroll
-                for (int e = 0; e < 4; ++e)
-                  if (4 * ng + e < valid) sq += yn[e] * yn[e];
-                if (full4) {
-                  *reinterpret_cast<float4 *>(y) = make_float4(yn[0], yn[1], yn[2], yn[3]);
-                  __nv_bfloat162 lo = __floats2bfloat162_rn(gn[0] * yn[0], gn[1] * yn[1]);
-                  __nv_bfloat162 hi = __floats2bfloat162_rn(gn[2] * yn[2], gn[3] * yn[3]);
-                  *reinterpret_cast<uint2 *>(p.xb + (size_t)t * p.ldo + col) = make_uint2(*(uint32_t *)&lo, *(uint32_t *)&hi);
-                } else {
-#pragma unroll
-                  for (int e = 0; e < 4; ++e)
-                    if (4 * ng + e < valid) {
-                      y[e] = yn[e];
-                      p.xb[(size_t)t * p.ldo + col + e] = __float2bfloat16_rn(gn[e] * yn[e]);
-                    }
-                }
-#pragma unroll
-                for (int o = 16; o; o >>= 1) sq += __shfl_xor_sync(0xffffffffu, sq, o);
-                if (lane == 0) p.ss_out[(size_t)tile * OURO_MAX_ROWS + t] = sq;
-              }
-              continue;
-            }
-            if (p.mode == MODE_QKV) {
-              const int cm = row0 + 4 * ng;                      // first of this thread's 4 columns inside q, k or v
-              const int half = p.head_dim >> 1;
-              const bool upper = (cm & half) != 0;
-              float4 cs4[4], sn4[4];
-#pragma unroll
-              for (int j = 0; j < 4; ++j) {
-                const int t = tb + j * n * 4;
-                cs4[j] = sn4[j] = make_float4(0.f, 0.f, 0.f, 0.f);
-                if (t < p.rows && seg != 2) {
-                  const size_t ti = (size_t)spos[t] * half + (cm & (half - 1));
-                  cs4[j] = *reinterpret_cast<const float4 *>(p.cos_t + ti);
-                  sn4[j] = *reinterpret_cast<const float4 *>(p.sin_t + ti);
-                }
-              }
-#pragma unroll
-              for (int j = 0; j < 4; ++j) {
-                const int t = tb + j * n * 4;
-                if (t >= p.rows) continue;                            // uniform inside the warp
-                const float r = rs[t];
-                const float vals[4] = {acc[j].x * r, acc[j].y * r, acc[j].z * r, acc[j].w * r};
-                float other[4];
-#pragma unroll
-                for (int e = 0; e < 4; ++e) other[e] = __shfl_xor_sync(0xffffffffu, vals[e], half >> 2);
-                const float cs[4] = {cs4[j].x, cs4[j].y, cs4[j].z, cs4[j].w}, sn[4] = {sn4[j].x, sn4[j].y, sn4[j].z, sn4[j].w};
-                float rv[4];
-#pragma unroll
-                for (int e = 0; e < 4; ++e)
-                  rv[e] = seg == 2 ? vals[e] : (upper ? vals[e] * cs[e] + other[e] * sn[e] : vals[e] * cs[e] - other[e] * sn[e]);
-                __nv_bfloat16 *dst = seg == 0 ? p.q_out + (size_t)t * p.dq + cm
-                                   : seg == 1 ? p.k_out + (size_t)(p.L + t) * p.dkv + cm
-                                              : p.v_out + (size_t)(p.L + t) * p.dkv + cm;
-                if (full4) {
-                  __nv_bfloat162 lo = __floats2bfloat162_rn(rv[0], rv[1]), hi = __floats2bfloat162_rn(rv[2], rv[3]);
-                  *reinterpret_cast<uint2 *>(dst) = make_uint2(*(uint32_t *)&lo, *(uint32_t *)&hi);
-                } else {
-#pragma unroll
-                  for (int e = 0; e < 4; ++e)
-                    if (4 * ng + e < valid) dst[e] = __float2bfloat16_rn(rv[e]);
-                }
-              }
-              continue;
-            }
-#pragma unroll
-            for (int j = 0; j < 4; ++j) {
-              const int t = tb + j * n * 4;
-              if (t >= p.rows) continue;                              // uniform inside the warp
-              const float r = rs[t];
-              const float vals[4] = {acc[j].x * r, acc[j].y * r, acc[j].z * r, acc[j].w * r};
-              if (p.mode == MODE_HEAD) {                              // the warp's 32 lanes hold the tile's 128 columns
-                uint32_t bu = 0;
-                int bi = col;
-#pragma unroll
-                for (int e = 0; e < 4; ++e) {
-                  uint32_t uo = ordered_u32(vals[e]);
-                  if (4 * ng + e < valid && uo > bu) { bu = uo; bi = col + e; }
-                }
-                const uint32_t mx = __reduce_max_sync(0xffffffffu, bu);
-                const int src_lane = __ffs(__ballot_sync(0xffffffffu, bu == mx)) - 1;   // lowest lane = smallest index
-                bi = __shfl_sync(0xffffffffu, bi, src_lane);
-                if (lane == 0) {
-                  p.tile_max[(size_t)tile * OURO_MAX_ROWS + t] = ordered_f32(mx);
-                  p.tile_arg[(size_t)tile * OURO_MAX_ROWS + t] = bi;
-                }
-              }
-              if (p.out_f32) {
-                float *y = p.out_f32 + (size_t)t * p.ldo + col;
-#pragma unroll
-                for (int e = 0; e < 4; ++e)
-                  if (4 * ng + e < valid) y[e] = p.mode == MODE_RESIDUAL ? y[e] + vals[e] : vals[e];
+                const int t = tb + j * js;
+                const bool in = c0 + cc < n && t < t_lim;
+                tg4[cc][j] = in ? __ldcg((const float4 *)(src + (size_t)t * TILE_N)) : make_float4(0.f, 0.f, 0.f, 0.f);
+                tu4[cc][j] = in ? __ldcg((const float4 *)(src + (size_t)t * TILE_N + 64)) : make_float4(0.f, 0.f, 0.f, 0.f);
               }
             }
+#pragma unroll
+            for (int cc = 0; cc < 4; ++cc)
+#pragma unroll
+              for (int j = 0; j < 4; ++j) {
+                g[j].x += tg4[cc][j].x; g[j].y += tg4[cc][j].y; g[j].z += tg4[cc][j].z; g[j].w += tg4[cc][j].w;
+                u[j].x += tu4[cc][j].x; u[j].y += tu4[cc][j].y; u[j].z += tu4[cc][j].z; u[j].w += tu4[cc][j].w;
+              }
           }
         }
-        epi_barrier();
-        if (et == 0) {                                                 // the last contributor to finish re-arms the tile
-          int d = atomicAdd(p.done + tile, 1);
-          if (d == n - 1) { p.counters[tile] = 0; p.done[tile] = 0; }
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          const int t = tb + j * js;
+          if (t < t_lim && feat < F) {
+            const float r = rs[t];
+            g[j].x *= r; g[j].y *= r; g[j].z *= r; g[j].w *= r;
+            u[j].x *= r; u[j].y *= r; u[j].z *= r; u[j].w *= r;
+            __nv_bfloat162 lo = __floats2bfloat162_rn(g[j].x / (1.0f + __expf(-g[j].x)) * u[j].x, g[j].y / (1.0f + __expf(-g[j].y)) * u[j].y);
+            __nv_bfloat162 hi = __floats2bfloat162_rn(g[j].z / (1.0f + __expf(-g[j].z)) * u[j].z, g[j].w / (1.0f + __expf(-g[j].w)) * u[j].w);
+            *(uint2 *)(p.out_bf16 + (size_t)t * F + feat) = make_uint2(*(uint32_t *)&lo, *(uint32_t *)&hi);
+          }
         }
       }
+      return true;
+    };
+
+    // Partial tiles.  Called once this CTA has published all its own partials, so waiting for the others cannot
+    // form a cycle.  The (at most two) tiles are finished side by side, each by one half of the epilogue threads.
+    auto run_fixups = [&]() {
+      const int grp = et >> 6, gi = et & 63;
+      bool mine = true;
+      if (grp < n_pend) {
+        const int tile = pend_tile[grp], n = pend_n[grp], first = pend_first[grp], my = (int)blockIdx.x - first;
+        mine = p.mode == MODE_SWIGLU ? finish_swiglu(tile, gi, 64, grp, my, n, first, nullptr, 0, p.rows)
+                                     : finish_plain(tile, gi, 64, grp, my, n, first, nullptr, 0, p.rows);
+        if (gi == 0 && grp == 0) TRACE(10);
+        if (mine) {
+          group_barrier(grp);
+          if (gi == 0) {                                               // the last contributor to finish re-arms the tile
+            int d = atomicAdd(p.done + tile, 1);
+            if (d == n - 1) { p.counters[tile] = 0; p.done[tile] = 0; }
+          }
+        }
+      }
+      if (gi == 0 && grp == 0) TRACE(11);
+      if (!mine) wait_flag[2] = 1;
+      epi_barrier();
+      if (wait_flag[2]) ok = false;
       n_pend = 0;
     };
 
@@ -587,6 +639,7 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_tc_kernel(const __grid_consta
       rs[et] = r;
       spos[et] = (p.mode == MODE_QKV && et < p.rows) ? p.pos[et] : 0;
     }
+    if (et == 0) wait_flag[2] = 0;
     epi_barrier();
 
     while (w.next(s)) {
@@ -603,130 +656,27 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_tc_kernel(const __grid_consta
       if (et == 0) TRACE(4);                       // overwritten per item: the last accumulator's arrival remains
       fence_after_sync();
       const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + a * acc_cols;
-      int seg = 0, row0 = 0, col0 = 0, valid = TILE_N;
-      if (p.mode != MODE_SWIGLU) locate(p, s.tile, seg, row0, col0, valid);
       if (s.n_contrib == 1) {
-        if (p.mode == MODE_SWIGLU) {
-          // rows 0..63 hold gate, rows 64..127 hold up, for output features tile*64 + (nl & 63)
-          const int F = p.a_rows[0];
-          const int feat = s.tile * 64 + (nl & 63);
-          for (int t0 = 0; t0 < p.t_pad; t0 += 16) {
+        // whole tile: the accumulators go to shared memory token-major, STAGE_TOK tokens at a time, and are finished
+        // from there; the TMEM buffer is handed back as soon as it has been read
+        for (int c0 = 0; c0 < p.t_pad; c0 += STAGE_TOK) {
+          const int c1 = min(p.t_pad, c0 + STAGE_TOK);
+          for (int t0 = c0; t0 < c1; t0 += 16) {
             tmem_ld16(taddr + t0, v);
 #pragma unroll
-            for (int i = 0; i < 16; ++i) v[i] *= rs[t0 + i];
-            if (nl >= 64) {
-#pragma unroll
-              for (int i = 0; i < 16; ++i) xchg[(t0 + i) * 64 + (nl - 64)] = v[i];
-            }
-            epi_barrier();
-            if (nl < 64 && feat < F) {
-#pragma unroll
-              for (int i = 0; i < 16; ++i) {
-                int t = t0 + i;
-                if (t < p.rows) {
-                  float g = v[i], u = xchg[t * 64 + nl];
-                  p.out_bf16[(size_t)t * F + feat] = __float2bfloat16_rn(g / (1.0f + __expf(-g)) * u);
-                }
-              }
-            }
-            epi_barrier();
+            for (int i = 0; i < 16; ++i) stage[(t0 - c0 + i) * TILE_N + nl] = v[i];
           }
-        } else {
-          float *xv = xchg;                                   // [4 quarters][128 tokens] best value
-          int *xi = (int *)(xchg + 4 * OURO_MAX_ROWS);        //                         and its index
-          for (int t0 = 0; t0 < p.t_pad; t0 += 16) {
-            tmem_ld16(taddr + t0, v);
-            if (p.mode == MODE_RESIDUAL && p.gain) {
-              // new residual stream, its bf16(gain * x) image for the next GEMM, and this tile's sums of squares
-              const float gcol = nl < valid ? __bfloat162float(p.gain[col0 + nl]) : 0.f;
-#pragma unroll
-              for (int i = 0; i < 16; ++i) {
-                const int t = t0 + i;
-                float y = 0.f;
-                if (t < p.rows && nl < valid) {
-                  float *yp = p.out_f32 + (size_t)t * p.ldo + col0 + nl;
-                  y = *yp + v[i];
-                  *yp = y;
-                  p.xb[(size_t)t * p.ldo + col0 + nl] = __float2bfloat16_rn(gcol * y);
-                }
-                float sq = y * y;
-#pragma unroll
-                for (int o = 16; o; o >>= 1) sq += __shfl_xor_sync(0xffffffffu, sq, o);
-                if (lane == 0) xv[q * OURO_MAX_ROWS + t] = sq;
-              }
-              continue;
-            }
-#pragma unroll
-            for (int i = 0; i < 16; ++i) v[i] *= rs[t0 + i];
-            if (p.mode == MODE_QKV) {
-              const int cm = row0 + nl;                          // column inside q, k or v
-              if (seg == 2) {
-                if (nl < valid)
-#pragma unroll
-                  for (int i = 0; i < 16; ++i)
-                    if (t0 + i < p.rows) p.v_out[(size_t)(p.L + t0 + i) * p.dkv + cm] = __float2bfloat16_rn(v[i]);
-              } else {
-                const int half = p.head_dim >> 1, ih = cm & (half - 1);
-                const bool upper = (cm & half) != 0;
-#pragma unroll
-                for (int i = 0; i < 16; ++i) xchg[i * TILE_N + nl] = v[i];
-                epi_barrier();
-                if (nl < valid) {
-#pragma unroll
-                  for (int i = 0; i < 16; ++i) {
-                    const int t = t0 + i;
-                    if (t < p.rows) {
-                      const float other = xchg[i * TILE_N + (nl ^ half)];
-                      const size_t ti = (size_t)spos[t] * half + ih;
-                      const float cs = p.cos_t[ti], sn = p.sin_t[ti];
-                      const float r = upper ? v[i] * cs + other * sn : v[i] * cs - other * sn;
-                      if (seg == 0) p.q_out[(size_t)t * p.dq + cm] = __float2bfloat16_rn(r);
-                      else p.k_out[(size_t)(p.L + t) * p.dkv + cm] = __float2bfloat16_rn(r);
-                    }
-                  }
-                }
-                epi_barrier();
-              }
-              continue;
-            }
-            store_chunk(p, col0 + nl, nl < valid, t0, v);
-            if (p.mode == MODE_HEAD) {
-#pragma unroll
-              for (int i = 0; i < 16; ++i) {
-                const uint32_t bu = nl < valid ? ordered_u32(v[i]) : 0u;
-                const uint32_t mx = __reduce_max_sync(0xffffffffu, bu);
-                const int src_lane = __ffs(__ballot_sync(0xffffffffu, bu == mx)) - 1;   // smallest index among equals
-                if (lane == 0) { xv[q * OURO_MAX_ROWS + t0 + i] = ordered_f32(mx); xi[q * OURO_MAX_ROWS + t0 + i] = col0 + q * 32 + src_lane; }
-              }
-            }
+          if (c1 == p.t_pad) {
+            fence_before_sync();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&acc_empty[a]);
           }
-          if (p.mode == MODE_RESIDUAL && p.gain) {
-            epi_barrier();
-            if (et < p.rows)
-              p.ss_out[(size_t)s.tile * OURO_MAX_ROWS + et] =
-                  ((xv[et] + xv[OURO_MAX_ROWS + et]) + xv[2 * OURO_MAX_ROWS + et]) + xv[3 * OURO_MAX_ROWS + et];
-            epi_barrier();
-          }
-          if (p.mode == MODE_HEAD) {
-            epi_barrier();
-            if (et < p.rows) {
-              float bv = xv[et];
-              int bi = xi[et];
-#pragma unroll
-              for (int qq = 1; qq < 4; ++qq) {
-                float ov = xv[qq * OURO_MAX_ROWS + et];
-                int oi = xi[qq * OURO_MAX_ROWS + et];
-                if (ov > bv || (ov == bv && oi < bi)) { bv = ov; bi = oi; }
-              }
-              p.tile_max[(size_t)s.tile * OURO_MAX_ROWS + et] = bv;
-              p.tile_arg[(size_t)s.tile * OURO_MAX_ROWS + et] = bi;
-            }
-            epi_barrier();
-          }
+          epi_barrier();
+          const int lim = min(c1, p.rows);
+          if (p.mode == MODE_SWIGLU) finish_swiglu(s.tile, et, 128, 0, 0, 1, 0, stage, c0, lim);
+          else finish_plain(s.tile, et, 128, 0, 0, 1, 0, stage, c0, lim);
+          epi_barrier();
         }
-        fence_before_sync();
-        __syncwarp();
-        if (lane == 0) mbar_arrive(&acc_empty[a]);
       } else {
         // partial tile: park it in this CTA's slot and announce it; the partials are added up after the loop
         float *mine = p.scratch + ((size_t)blockIdx.x * 2 + s.slot) * SLOT_FLOATS;
@@ -750,7 +700,7 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_tc_kernel(const __grid_consta
       ++item;
     }
     if (et == 0) TRACE(5);
-    run_fixups();
+    if (ok) run_fixups();
     if (et == 0) TRACE(7);
     if (!ok && et == 0) { *abort_flag = 1; atomicExch(p.status, 1); }
   }

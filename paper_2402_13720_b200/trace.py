@@ -66,6 +66,7 @@ def main():
     names = ["q,k,v", "o-proj", "gate,up", "down", "LM head"]
     points = [(0, "CTA entry"), (8, "last weight load issued"), (2, "first stage full"), (3, "last MMA issued"),
               (4, "last accumulator complete"), (5, "whole tiles done / fix-up begins"), (6, "partials of the others there"),
+              (9, "  group 0: past the wait + fence"), (10, "  group 0: its tokens finished"), (11, "  group 0: tile re-armed"),
               (7, "fix-up done")]
     spans = []
     for kind in range(5):
