@@ -156,7 +156,10 @@ int ouro_pool_import(ouro_ctx *ctx, const int32_t *ngrams_host, int32_t n);
 /* Eq. 7: packs [pending, d_1..d_gamma, p^1_2..beta, .., p^K'_2..beta] into the target's query block with
  * position ids (trunk row b: L+b; suffix row (j,i): L+gamma+i) and the Eq. 8 visibility.  draft_dev
  * [gamma].  suffix_dev / count_dev as written by ouro_phrase_lookup; pass NULL for both to have the
- * pool looked up with key d_gamma here.  Synchronises (the row count is needed on the host). */
+ * pool looked up with key d_gamma here.  Asynchronous when the target runs on the tensor-core kernels (bf16,
+ * supported shapes): the block's row count 1 + gamma + K' (beta-1) then stays on the device, the forward is
+ * launched for the largest block the parameters allow and ouro_block_get reports the true count.  Otherwise the
+ * call synchronises to read the count. */
 int ouro_assemble_candidates(ouro_ctx *ctx, const int32_t *draft_dev, const int32_t *suffix_dev,
                              const int32_t *count_dev);
 /* Plain causal block of n tokens (tokens_dev [n]) for model `which`: prefill, catch-up, vanilla decoding. */
@@ -206,7 +209,10 @@ int ouro_generate_vanilla(ouro_ctx *ctx, const int32_t *prompt_host, int32_t n_p
 enum {
   OURO_PROF_OFF = -1, OURO_PROF_EMBED = 0, OURO_PROF_NORM = 1, OURO_PROF_QKV = 2, OURO_PROF_ROPE = 3,
   OURO_PROF_ATTENTION = 4, OURO_PROF_WO = 5, OURO_PROF_GATEUP = 6, OURO_PROF_DOWN = 7, OURO_PROF_HEAD = 8,
-  OURO_PROF_ARGMAX = 9, OURO_PROF_FORWARD = 10 /* the whole forward */
+  OURO_PROF_ARGMAX = 9, OURO_PROF_FORWARD = 10 /* the whole forward */,
+  OURO_PROF_GEMM = 11 /* every launch of the weight-streaming GEMM kernel; consecutive GEMMs (output projection, gate/up,
+                         down, the next q,k,v or the LM head) run as ONE launch, except while one of the classes
+                         QKV..HEAD is being timed: then each GEMM is launched alone so that it can be */
 };
 /* Number of kernels this library has launched in this process (all contexts), for launch accounting. */
 uint64_t ouro_kernel_launches(void);

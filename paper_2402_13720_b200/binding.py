@@ -322,7 +322,7 @@ class Engine:
         self._ck(self.L.ouro_advance(self.ctx, which, n))
 
     # ---- measurement -------------------------------------------------------------------------
-    PROF = dict(off=-1, embed=0, norm=1, qkv=2, rope=3, attention=4, wo=5, gateup=6, down=7, head=8, argmax=9, forward=10)
+    PROF = dict(off=-1, embed=0, norm=1, qkv=2, rope=3, attention=4, wo=5, gateup=6, down=7, head=8, argmax=9, forward=10, gemm=11)
 
     def profile_enable(self, kernel_class):
         self._ck(self.L.ouro_profile_enable(self.ctx, self.PROF[kernel_class] if isinstance(kernel_class, str) else kernel_class))

@@ -174,6 +174,9 @@ static bool mem_ok(const ouro_model_mem *m) {
 }
 
 int ouro_fast_setup(ouro_ctx *c);  // tensor maps etc. of the tensor-core paths (gemm_tc.cu)
+void ouro_fast_reset(ouro_ctx *c, bool force);   // clears split-K / chain counters (always, or only after a device-side give-up)
+void ouro_fast_mark_dirty(ouro_ctx *c);
+bool ouro_fast_available(ouro_ctx *c, int which);   // model `which` runs on the tensor-core kernels
 
 extern "C" int ouro_create(const ouro_model_desc *t, const ouro_model_mem *tm, const ouro_model_desc *d,
                            const ouro_model_mem *dm, const ouro_params *p, void *ws, size_t ws_bytes, void *stream,
@@ -269,6 +272,7 @@ extern "C" int ouro_reset(ouro_ctx *c, int keep_pool) {
   forget_blocks(c);
   c->seq.assign(1, 0);
   c->step = 0;
+  ouro_fast_reset(c, true);
   launch_set_state(c->st, c->seq_dev, 1, 0, 1, c->stream);
   if (!keep_pool) launch_pool_clear(c->pool, c->st, c->stream);
   CKL();
@@ -285,6 +289,7 @@ extern "C" int ouro_set_state(ouro_ctx *c, int32_t cache_len, int32_t pending) {
   c->seq.assign((size_t)cache_len + 1, 0);
   c->seq.back() = pending;
   c->step = 0;
+  ouro_fast_reset(c, false);
   launch_set_state(c->st, c->seq_dev, cache_len + 1, pending, 1, c->stream);
   CKL();
   return OURO_OK;
@@ -315,6 +320,7 @@ extern "C" int ouro_assemble_causal(ouro_ctx *c, int which, const int32_t *token
   launch_assemble_causal(M.blk, tokens_dev, n, M.L, c->stream);
   CKL();
   M.blk_rows = n;
+  M.blk_rows_dev = false;
   M.blk_L = M.L;
   M.blk_is_candidate = false;
   return OURO_OK;
@@ -342,23 +348,22 @@ extern "C" int ouro_assemble_candidates(ouro_ctx *c, const int32_t *draft_dev, c
   ModelRt &M = c->m[OURO_TARGET];
   const int gamma = c->p.gamma, S = c->p.beta - 1, K = c->p.K;
   if (M.L + 1 + gamma + K * S > M.d.max_seq) return fail(c, OURO_ECAPACITY, "cache length + block rows exceeds max_seq");
-  if (!suffix_dev && c->mbox) {
-    const int32_t seq = ++c->mseq;
-    launch_lookup_assemble(c->pool, M.blk, c->st, draft_dev, c->cand_suffix, c->cand_count, M.L, gamma, S, K, c->mbox_dev, seq,
+  if (!suffix_dev)
+    launch_lookup_assemble(c->pool, M.blk, c->st, draft_dev, c->cand_suffix, c->cand_count, M.L, gamma, S, K, nullptr, 0,
                            c->stream);
-    CKL();
-    TRY(mbox_wait(c, MBOX_ROWS, seq));
-    M.blk_rows = c->mbox[MBOX_ROWS + 1];
+  else
+    launch_assemble_candidates(M.blk, c->st, draft_dev, suffix_dev, count_dev, M.L, gamma, S, K, c->stream);
+  CKL();
+  if (ouro_fast_available(c, OURO_TARGET)) {
+    // The tensor-core kernels read the block's row count from device memory: the forward is launched for the largest
+    // block these parameters allow and the host never waits for the lookup.
+    M.blk_rows = 1 + gamma + K * S;
+    M.blk_rows_dev = true;
   } else {
-    if (!suffix_dev)
-      launch_lookup_assemble(c->pool, M.blk, c->st, draft_dev, c->cand_suffix, c->cand_count, M.L, gamma, S, K, nullptr, 0,
-                             c->stream);
-    else
-      launch_assemble_candidates(M.blk, c->st, draft_dev, suffix_dev, count_dev, M.L, gamma, S, K, c->stream);
-    CKL();
     CK(cudaMemcpyAsync(c->pin, &c->st->n_rows, sizeof(int32_t), cudaMemcpyDeviceToHost, c->stream));
     CK(cudaStreamSynchronize(c->stream));
     M.blk_rows = c->pin[0];
+    M.blk_rows_dev = false;
   }
   M.blk_L = M.L;
   M.blk_is_candidate = true;
@@ -370,8 +375,15 @@ extern "C" int ouro_block_get(ouro_ctx *c, int which, int32_t *tok, int32_t *pos
   if (!c || which < 0 || which > 1) return OURO_EINVAL;
   ModelRt &M = c->m[which];
   if (!M.present || M.blk_rows == 0) return fail(c, OURO_ESTATE, "no block assembled");
-  size_t n = M.blk_rows;
   CK(cudaStreamSynchronize(c->stream));
+  if (M.blk_rows_dev) {                      // the host only knows an upper bound so far
+    int32_t exact = 0;
+    CK(cudaMemcpy(&exact, &c->st->n_rows, sizeof(int32_t), cudaMemcpyDeviceToHost));
+    if (exact < 1 || exact > M.blk_rows) return fail(c, OURO_ECUDA, "block has an impossible row count");
+    M.blk_rows = exact;
+    M.blk_rows_dev = false;
+  }
+  size_t n = M.blk_rows;
   if (tok) CK(cudaMemcpy(tok, M.blk.tok, n * 4, cudaMemcpyDeviceToHost));
   if (pos) CK(cudaMemcpy(pos, M.blk.pos, n * 4, cudaMemcpyDeviceToHost));
   if (group) CK(cudaMemcpy(group, M.blk.group, n * 4, cudaMemcpyDeviceToHost));
@@ -404,7 +416,7 @@ void prof_mark(ouro_ctx *c, int) {
   cudaEventRecord(c->prof_ev[c->prof_used++], c->stream);
 }
 extern "C" int ouro_profile_enable(ouro_ctx *c, int kernel_class) {
-  if (!c || kernel_class < OURO_PROF_OFF || kernel_class > OURO_PROF_FORWARD) return OURO_EINVAL;
+  if (!c || kernel_class < OURO_PROF_OFF || kernel_class > OURO_PROF_GEMM) return OURO_EINVAL;
   prof_flush(c);
   c->prof_class = kernel_class;
   c->prof_ms = 0.0;
@@ -434,6 +446,7 @@ static int forward(ouro_ctx *c, int which, int32_t *argmax_dev, float *logits_de
   cudaStream_t s = c->stream;
   Activations &a = c->a;
   ProfScope whole(c, OURO_PROF_FORWARD);
+  c->cur_rows_dev = M.blk_rows_dev ? &c->st->n_rows : nullptr;
   if (ouro_fast_embed(c, which, rows) == OURO_ESTATE) {
     ProfScope ps(c, OURO_PROF_EMBED);
     launch_embed(dt, M.embed, M.blk.tok, rows, d.d_model, a.x, s);
@@ -589,6 +602,7 @@ struct AcceptOut {
   int32_t A, chosen, m, n_acc;
   int32_t accepted[OURO_MAX_GAMMA + OURO_MAX_BETA];
   int32_t status;
+  int32_t n_cand;     // candidates the block held (K' <= K)
 };
 
 static int accept_step(ouro_ctx *c, const int32_t *argmax_dev, AcceptOut *r) {
@@ -598,7 +612,7 @@ static int accept_step(ouro_ctx *c, const int32_t *argmax_dev, AcceptOut *r) {
   const int gamma = c->p.gamma, S = c->p.beta - 1, L = T.L;
   cudaStream_t s = c->stream;
   static_assert(sizeof(AcceptOut) <= PIN_INTS * 4, "pinned staging too small");
-  static_assert(sizeof(AcceptOut) == (4 + OURO_MAX_GAMMA + OURO_MAX_BETA + 1) * 4 && MBOX_ACCEPT + 1 + sizeof(AcceptOut) / 4 <= MBOX_INTS,
+  static_assert(sizeof(AcceptOut) == (4 + OURO_MAX_GAMMA + OURO_MAX_BETA + 2) * 4 && MBOX_ACCEPT + 1 + sizeof(AcceptOut) / 4 <= MBOX_INTS,
                 "acceptance record and mailbox slot disagree");
   if (c->mbox) {
     const int32_t seq = ++c->mseq;
@@ -615,7 +629,10 @@ static int accept_step(ouro_ctx *c, const int32_t *argmax_dev, AcceptOut *r) {
     CK(cudaStreamSynchronize(s));
     memcpy(r, c->pin, sizeof(AcceptOut));
   }
-  if (r->status != 0) return fail(c, OURO_ETIMEOUT, "device status word " + std::to_string(r->status));
+  if (r->status != 0) {
+    ouro_fast_mark_dirty(c);
+    return fail(c, OURO_ETIMEOUT, "device status word " + std::to_string(r->status));
+  }
   if (r->n_acc < 1 || r->n_acc > gamma + S + 1) return fail(c, OURO_ECUDA, "acceptance returned an impossible count");
   c->seq.insert(c->seq.end(), r->accepted, r->accepted + r->n_acc);
   T.L = L + r->n_acc;
@@ -665,6 +682,7 @@ static int draft_step_phrases(ouro_ctx *c, int32_t *out_dev, int *calls) {
     CK(cudaMemcpyAsync(c->pin, &c->st->n_rows, sizeof(int32_t), cudaMemcpyDeviceToHost, s));
     CK(cudaStreamSynchronize(s));
     D.blk_rows = c->pin[0];
+    D.blk_rows_dev = false;
     D.blk_L = D.L;
     D.blk_is_candidate = true;
     if (D.blk_rows < n || D.blk_rows > n + K * S) return fail(c, OURO_ECUDA, "draft block has an impossible row count");
@@ -743,7 +761,6 @@ extern "C" int ouro_generate(ouro_ctx *c, const int32_t *prompt, int32_t n_promp
     TRY(draft_step(c, c->draft_dev, &st.draft_calls));
     CK(cudaEventRecord(c->ev[2], s));
     TRY(ouro_assemble_candidates(c, c->draft_dev, nullptr, nullptr));
-    st.candidates += (T.blk_rows - 1 - gamma) / std::max(1, S);
     CK(cudaEventRecord(c->ev[3], s));
     TRY(forward(c, OURO_TARGET, c->a.argmax, nullptr));
     CK(cudaEventRecord(c->ev[4], s));
@@ -758,6 +775,7 @@ extern "C" int ouro_generate(ouro_ctx *c, const int32_t *prompt, int32_t n_promp
     st.target_calls += 1;
     st.full_accepts += r.A == gamma;
     st.suffix_tokens += r.chosen >= 0 ? r.m : 0;
+    st.candidates += r.n_cand;
     for (int i = 0; i < r.n_acc && n < max_new; ++i) {
       out[n++] = r.accepted[i];
       if (c->p.eos_token >= 0 && r.accepted[i] == c->p.eos_token) { stop = true; break; }

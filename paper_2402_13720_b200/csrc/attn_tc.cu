@@ -41,6 +41,7 @@ struct AttnParams {
   float *part;                     // [rows][H][cap][HD+2]: max (log2 domain), sum, unnormalised output
   __nv_bfloat16 *out;              // [rows][H*HD]
   int direct;                      // every row's keys lie in span 0: the span kernel normalises and writes `out` itself
+  const int *rows_dev;             // NULL, or the block's true row count in device memory (`rows` is then an upper bound)
 };
 
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -124,15 +125,16 @@ __global__ void __launch_bounds__(THREADS) attn_span_kernel(const AttnParams p) 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int sc = blockIdx.x, kvh = blockIdx.y;
   const int g = p.H / p.Hkv, dkv = p.Hkv * HD;
-  const int M_all = g * p.rows;
+  const int rows = p.rows_dev ? min(p.rows, __ldg(p.rows_dev)) : p.rows;   // written before the forward pass began
+  const int M_all = g * rows;
 
   int nv_max = 0;
-  for (int r = threadIdx.x; r < p.rows; r += THREADS) {
+  for (int r = threadIdx.x; r < rows; r += THREADS) {
     s_nvis[r] = p.lin_end[r] + p.seg_len[r];
     s_grp[r] = p.group[r];
   }
   __syncthreads();
-  for (int r = 0; r < p.rows; ++r) nv_max = max(nv_max, s_nvis[r]);
+  for (int r = 0; r < rows; ++r) nv_max = max(nv_max, s_nvis[r]);
   const int span0 = sc * SPAN;
   const int n_chunks = min(SC, (nv_max - span0 + CH - 1) / CH);       // chunks of this span anybody sees
 
@@ -162,7 +164,7 @@ __global__ void __launch_bounds__(THREADS) attn_span_kernel(const AttnParams p) 
     // in row tile mt: lane/4 and +8.
     if (threadIdx.x < QR) {
       int r0 = 0, hq = 0;
-      if (m0 + (int)threadIdx.x < M_all) map_row(m0 + threadIdx.x, g, p.rows, s_grp, r0, hq);
+      if (m0 + (int)threadIdx.x < M_all) map_row(m0 + threadIdx.x, g, rows, s_grp, r0, hq);
       s_map[threadIdx.x] = r0 | (hq << 16);
     }
     __syncthreads();
@@ -209,13 +211,13 @@ __global__ void __launch_bounds__(THREADS) attn_span_kernel(const AttnParams p) 
       __syncthreads();
       const bool common = c0 + CH <= p.L;
       int g_begin = 0;
-      while (g_begin < p.rows) {
+      while (g_begin < rows) {
         // -------------------------------------------------------------- one pass over the chunk
-        int g_end = p.rows, gid = -2;                  // gid -2: every row takes part
+        int g_end = rows, gid = -2;                  // gid -2: every row takes part
         if (!common) {
           gid = s_grp[g_begin];
           g_end = g_begin + 1;
-          while (g_end < p.rows && s_grp[g_end] == gid) ++g_end;
+          while (g_end < rows && s_grp[g_end] == gid) ++g_end;
           const int last = g_end - 1, nvg = s_nvis[last];
           int lin_g = INT_MAX, seg_g = 0;
           if (p.seg_len[last] > 0) { lin_g = p.lin_end[last]; seg_g = p.seg_start[last]; }
@@ -402,7 +404,7 @@ __global__ void attn_merge_kernel(const AttnParams p) {
   pdl_wait();
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int r = blockIdx.x, head = blockIdx.y * (blockDim.x >> 5) + warp;
-  if (head >= p.H) return;
+  if (head >= p.H || (p.rows_dev && r >= __ldg(p.rows_dev))) return;
   const int nv = p.lin_end[r] + p.seg_len[r];
   const int ns = (nv + SPAN - 1) / SPAN;
   const float *src = p.part + ((size_t)r * p.H + head) * p.cap * PW;
@@ -446,9 +448,11 @@ int attention_tc_setup() {
 }
 
 // Folds the per-span pieces written by either span kernel (head dim 64 or 128) into the block's attention output.
-void launch_attention_merge(const ouro_model_desc &d, const BlockDev &b, int rows, float *part, void *out, cudaStream_t s) {
+void launch_attention_merge(const ouro_model_desc &d, const BlockDev &b, int rows, float *part, void *out, const int *rows_dev,
+                            cudaStream_t s) {
   OURO_COUNT_LAUNCH();
   AttnParams p{};
+  p.rows_dev = rows_dev;
   p.lin_end = b.lin_end; p.seg_start = b.seg_start; p.seg_len = b.seg_len; p.group = b.group;
   p.rows = rows; p.H = d.n_heads; p.Hkv = d.n_kv_heads;
   p.cap = (d.max_seq + SPAN - 1) / SPAN;
@@ -463,9 +467,10 @@ void launch_attention_merge(const ouro_model_desc &d, const BlockDev &b, int row
 
 // n_vis_max: an upper bound of the number of keys any row of the block sees (cache length + rows).
 void launch_attention_tc(const ouro_model_desc &d, const void *q, const void *k_cache, const void *v_cache, const BlockDev &b,
-                         int rows, int L, int n_vis_max, int layer, float *part, void *out, cudaStream_t s) {
+                         int rows, int L, int n_vis_max, int layer, float *part, void *out, const int *rows_dev, cudaStream_t s) {
   OURO_COUNT_LAUNCH();
   AttnParams p;
+  p.rows_dev = rows_dev;
   size_t off = (size_t)layer * d.max_seq * d.n_kv_heads * d.head_dim;
   p.q = (const __nv_bfloat16 *)q;
   p.k = (const __nv_bfloat16 *)k_cache + off;

@@ -70,7 +70,9 @@ struct GemmParams {
   int tiles;          // total tiles
   int kb;             // k-blocks per tile (K / 64)
   int t_pad;          // tokens padded to a multiple of 16 (MMA N)
-  int rows;           // valid tokens
+  int rows;           // valid tokens (an upper bound when rows_dev is set)
+  const int *rows_dev;  // NULL, or where the block's true row count sits in device memory: the host then sizes the
+                        // launch for the largest block the decoding parameters allow and never reads the count
   int stages;
   float *out_f32;     // MODE_STORE / MODE_RESIDUAL: [rows, ldo]
   int ldo;
@@ -98,6 +100,20 @@ struct GemmParams {
   int *status;        // context status word
   int trace_id;           // which GEMM of the layer this is (timeline builds only)
 };
+
+// A chain of GEMMs run by one persistent launch, each consuming what the one before produced (output projection ->
+// gate/up -> down -> next layer's q,k,v or the LM head).  The weight producer runs straight on into the next GEMM's
+// tiles; the activations of GEMM i + 1 are fetched once GEMM i has finished all its tiles, which the CTAs learn from
+// a counter in global memory (one per chain position, counting finished tiles, never reset: the host passes the value
+// it will have reached).  All GEMMs of a chain have the same rows / t_pad / stages.
+constexpr int MAX_CHAIN = 4;
+struct ChainParams {
+  GemmParams g[MAX_CHAIN];
+  int n;
+  int *finished;            // [MAX_CHAIN] tiles finished, per chain position (monotonic)
+  int target[MAX_CHAIN];    // value finished[i] has when GEMM i of this launch is complete
+};
+static_assert(sizeof(ChainParams) <= 4096, "kernel parameters");
 
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
@@ -171,10 +187,14 @@ __device__ __forceinline__ uint32_t ordered_u32(float f) {
 __device__ __forceinline__ float ordered_f32(uint32_t u) {
   return __uint_as_float((u & 0x80000000u) ? (u & 0x7fffffffu) : ~u);
 }
+// x * sigmoid(x) with the fast exponential and reciprocal (the result is rounded to bf16 right after)
+__device__ __forceinline__ float silu(float x) { return __fdividef(x, 1.0f + __expf(-x)); }
 __device__ __forceinline__ void epi_barrier() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
 // one half (64 threads) of the epilogue warps; grp = 0 or 1
 __device__ __forceinline__ void group_barrier(int grp) { asm volatile("bar.sync %0, 64;" ::"r"(2 + grp) : "memory"); }
-constexpr int STAGE_TOK = 64;     // tokens of a whole tile parked in shared memory at a time (64 x 128 fp32 = 32 KB)
+constexpr int STAGE_TOK = 64;     // tokens of a whole tile parked in shared memory at a time
+constexpr int STAGE_PITCH = TILE_N + 4;   // floats per parked token: 16-byte aligned rows that start 4 banks apart
+constexpr int STAGE_BYTES = STAGE_TOK * STAGE_PITCH * 4;
 
 // The schedule of this launch for CTA blockIdx.x (see weight_stream.cuh).
 struct SpanWalker : ws::SpanWalker {
@@ -196,14 +216,26 @@ __device__ __forceinline__ void locate(const GemmParams &p, int tile, int &seg, 
   valid = min(TILE_N, p.a_rows[seg] - row0);
 }
 
-__global__ void __launch_bounds__(THREADS, 1) gemm_tc_kernel(const __grid_constant__ GemmParams p) {
+// Bounded wait until GEMM `i` of the chain has finished all its tiles (acquire).
+__device__ __forceinline__ bool chain_wait(const ChainParams &cp, int i) {
+  for (uint32_t spin = 0; spin < (1u << 22); ++spin) {
+    int seen;
+    asm volatile("ld.acquire.gpu.global.b32 %0, [%1];" : "=r"(seen) : "l"(cp.finished + i) : "memory");
+    if (seen - cp.target[i] >= 0) return true;
+  }
+  return false;
+}
+
+__global__ void __launch_bounds__(THREADS, 1) gemm_tc_kernel(const __grid_constant__ ChainParams cp) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t *smem = (uint8_t *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
-  const int b_bytes = p.t_pad * BLOCK_K * 2;
+  const GemmParams &p0 = cp.g[0];                 // rows, t_pad and stages are common to the chain
+  const int n_stages = p0.stages;
+  const int b_bytes = p0.t_pad * BLOCK_K * 2;
   const int stage_bytes = A_BYTES + b_bytes;
   uint8_t *ring = smem;
-  float *xchg = (float *)(ring + (size_t)p.stages * stage_bytes);          // [64 tokens][128] accumulators of a whole tile
-  uint64_t *bars = (uint64_t *)((uint8_t *)xchg + 64 * OURO_MAX_ROWS * 4);
+  float *xchg = (float *)(ring + (size_t)n_stages * stage_bytes);          // [64 tokens][128] accumulators of a whole tile
+  uint64_t *bars = (uint64_t *)((uint8_t *)xchg + STAGE_BYTES);
   uint64_t *full = bars, *empty = bars + 16, *acc_full = bars + 32, *acc_empty = bars + 34;
   uint32_t *tmem_base_p = (uint32_t *)(bars + 36);
   volatile int *abort_flag = (volatile int *)(bars + 37);
@@ -212,12 +244,12 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_tc_kernel(const __grid_consta
   int *spos = (int *)(rs + OURO_MAX_ROWS);                  // [128] token positions (rotary table rows), QKV epilogue
 
   pdl_trigger();
-  if (threadIdx.x == 0) TRACE(0);
+  if (threadIdx.x == 0) { const GemmParams &p = p0; TRACE(0); }
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int acc_cols = p.t_pad <= 32 ? 32 : p.t_pad <= 64 ? 64 : 128;   // columns per accumulator buffer
+  const int acc_cols = p0.t_pad <= 32 ? 32 : p0.t_pad <= 64 ? 64 : 128;   // columns per accumulator buffer
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < p.stages; ++s) {
+    for (int s = 0; s < n_stages; ++s) {
       mbar_init(&full[s], 2);          // weight producer + activation producer, each with its byte count
       mbar_init(&empty[s], 1);
     }
@@ -243,6 +275,10 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_tc_kernel(const __grid_consta
     if (lane == 0) {
       // The weights do not depend on the previous kernel, so this warp never waits for it: the ring fills with
       // weight tiles while the predecessor drains.  The activation tiles come from warp 6, after its wait.
+      uint32_t n = 0;
+      bool ok = true;
+      for (int ci = 0; ci < cp.n && ok; ++ci) {
+      const GemmParams &p = cp.g[ci];
       auto issue = [&](const Span &s, int kb, int st) {
         uint8_t *sa = ring + (size_t)st * stage_bytes;
         mbar_expect_tx(&full[st], A_BYTES);
@@ -257,47 +293,59 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_tc_kernel(const __grid_consta
       };
       SpanWalker w(p);
       Span s;
-      uint32_t n = 0;
-      bool ok = true;
       while (ok && w.next(s)) {
         for (int kb = s.kb0; kb < s.kb1 && ok; ++kb, ++n) {
-          int st = n % p.stages;
-          if (n >= (uint32_t)p.stages) ok = mbar_wait(&empty[st], ((n / p.stages) - 1) & 1) && !*abort_flag;
+          int st = n % n_stages;
+          if (n >= (uint32_t)n_stages) ok = mbar_wait(&empty[st], ((n / n_stages) - 1) & 1) && !*abort_flag;
           if (!ok) break;
           issue(s, kb, st);
         }
       }
       TRACE(8);
-      if (!ok) { *abort_flag = 1; atomicExch(p.status, 1); }
+      }
+      if (!ok) { *abort_flag = 1; atomicExch(p0.status, 1); }
     }
   } else if (warp == 6) {
     // ---------------------------------------------------------------- activation producer
     if (lane == 0) {
-      pdl_wait();                                  // the activations are the previous kernel's output
-      TRACE(1);
-      SpanWalker w(p);
-      Span s;
+      pdl_wait();                                  // the first GEMM's activations are the previous kernel's output
       uint32_t n = 0;
       bool ok = true;
-      while (ok && w.next(s)) {
-        for (int kb = s.kb0; kb < s.kb1 && ok; ++kb, ++n) {
-          int st = n % p.stages;
-          if (n >= (uint32_t)p.stages) ok = mbar_wait(&empty[st], ((n / p.stages) - 1) & 1) && !*abort_flag;
+      for (int ci = 0; ci < cp.n && ok; ++ci) {
+        const GemmParams &p = cp.g[ci];
+        if (ci > 0) {
+          // they are what the GEMM before this one wrote: wait until all its tiles are finished, then make
+          // those generic-proxy writes visible to the copy engine's reads
+          ok = chain_wait(cp, ci - 1) && !*abort_flag;
           if (!ok) break;
-          mbar_expect_tx(&full[st], b_bytes);
-          tma_load_2d(ring + (size_t)st * stage_bytes + A_BYTES, &p.b, &full[st], kb * BLOCK_K, 0, HINT_EVICT_LAST);
+          asm volatile("fence.proxy.async;" ::: "memory");
+        }
+        TRACE(1);
+        SpanWalker w(p);
+        Span s;
+        while (ok && w.next(s)) {
+          for (int kb = s.kb0; kb < s.kb1 && ok; ++kb, ++n) {
+            int st = n % n_stages;
+            if (n >= (uint32_t)n_stages) ok = mbar_wait(&empty[st], ((n / n_stages) - 1) & 1) && !*abort_flag;
+            if (!ok) break;
+            mbar_expect_tx(&full[st], b_bytes);
+            tma_load_2d(ring + (size_t)st * stage_bytes + A_BYTES, &p.b, &full[st], kb * BLOCK_K, 0, HINT_EVICT_LAST);
+          }
         }
       }
-      if (!ok) { *abort_flag = 1; atomicExch(p.status, 1); }
+      if (!ok) { *abort_flag = 1; atomicExch(p0.status, 1); }
     }
   } else if (warp == 1) {
     // ---------------------------------------------------------------- MMA issuer
     if (lane == 0) {
-      const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(p.t_pad >> 3) << 17) | ((uint32_t)(TILE_N >> 4) << 24);
-      SpanWalker w(p);
-      Span s;
+      const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(p0.t_pad >> 3) << 17) | ((uint32_t)(TILE_N >> 4) << 24);
       uint32_t n = 0, item = 0;
       bool ok = true;
+      for (int ci = 0; ci < cp.n && ok; ++ci) {
+      const GemmParams &p = cp.g[ci];
+      SpanWalker w(p);
+      Span s;
+      bool first = true;
       while (ok && w.next(s)) {
         int a = item & 1;
         if (item >= 2) ok = mbar_wait(&acc_empty[a], ((item >> 1) - 1) & 1) && !*abort_flag;
@@ -305,10 +353,10 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_tc_kernel(const __grid_consta
         fence_after_sync();
         uint32_t tmem_d = tmem_base + a * acc_cols;
         for (int kb = s.kb0; kb < s.kb1; ++kb, ++n) {
-          int st = n % p.stages;
-          ok = mbar_wait(&full[st], (n / p.stages) & 1) && !*abort_flag;
+          int st = n % n_stages;
+          ok = mbar_wait(&full[st], (n / n_stages) & 1) && !*abort_flag;
           if (!ok) break;
-          if (n == 0) TRACE(2);
+          if (first) { TRACE(2); first = false; }
           fence_after_sync();
           uint32_t sa = smem_u32(ring + (size_t)st * stage_bytes), sb = sa + A_BYTES;
           uint64_t da = smem_desc_sw128(sa), db = smem_desc_sw128(sb);
@@ -321,7 +369,8 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_tc_kernel(const __grid_consta
         ++item;
       }
       TRACE(3);
-      if (!ok) { *abort_flag = 1; atomicExch(p.status, 1); }
+      }
+      if (!ok) { *abort_flag = 1; atomicExch(p0.status, 1); }
     }
   } else {
     // ---------------------------------------------------------------- epilogue warps
@@ -329,13 +378,17 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_tc_kernel(const __grid_consta
     const int q = warp & 3;                      // TMEM lane quarter this warp may read
     const int nl = q * 32 + lane;                // row of the tile held by this thread
     const int et = threadIdx.x - 64;             // 0..127 among the epilogue threads
-    SpanWalker w(p);
-    Span s;
     uint32_t item = 0;
     bool ok = true;
     float v[16];
+    for (int ci = 0; ci < cp.n && ok; ++ci) {
+    const GemmParams &p = cp.g[ci];
+    const bool publish = ci + 1 < cp.n;          // a later GEMM of the chain consumes this one's output
+    const int rows = p.rows_dev ? min(p.rows, __ldg(p.rows_dev)) : p.rows;
+    SpanWalker w(p);
+    Span s;
     int pend_tile[2], pend_n[2], pend_first[2], n_pend = 0;     // partial tiles this CTA contributed to (<= 2)
-    float *stage = xchg;                                         // [STAGE_TOK tokens][128 tile rows] fp32
+    float *stage = xchg;                                         // [STAGE_TOK tokens][STAGE_PITCH] fp32, 128 tile rows each
 
     // Finishing tokens of a tile.  Whatever produced the accumulator values - this CTA's own whole tile, parked
     // in shared memory token-major, or the partial tiles of all contributors in scratch - the last step is the
@@ -415,7 +468,7 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_tc_kernel(const __grid_consta
 #pragma unroll
           for (int j = 0; j < 4; ++j) {
             const int t = tb + j * js;
-            acc[j] = t < t_lim ? *reinterpret_cast<const float4 *>(stg + (size_t)(t - t_base) * TILE_N + 4 * ng)
+            acc[j] = t < t_lim ? *reinterpret_cast<const float4 *>(stg + (size_t)(t - t_base) * STAGE_PITCH + 4 * ng)
                                : make_float4(0.f, 0.f, 0.f, 0.f);
           }
         } else {
@@ -508,7 +561,7 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_tc_kernel(const __grid_consta
           if (t >= t_lim) continue;                                  // uniform inside the warp
           const float r = rs[t];
           const float vals[4] = {acc[j].x * r, acc[j].y * r, acc[j].z * r, acc[j].w * r};
-          if (p.mode == MODE_HEAD) {                                 // the warp's 32 lanes hold the tile's 128 columns
+          if (p.mode == MODE_HEAD && !stg) {                         // the warp's 32 lanes hold the tile's 128 columns
             uint32_t bu = 0;
             int bi = col;
 #pragma unroll
@@ -558,8 +611,8 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_tc_kernel(const __grid_consta
             const int t = tb + j * js;
             g[j] = u[j] = make_float4(0.f, 0.f, 0.f, 0.f);
             if (t < t_lim) {
-              g[j] = *reinterpret_cast<const float4 *>(stg + (size_t)(t - t_base) * TILE_N + 4 * ng);
-              u[j] = *reinterpret_cast<const float4 *>(stg + (size_t)(t - t_base) * TILE_N + 64 + 4 * ng);
+              g[j] = *reinterpret_cast<const float4 *>(stg + (size_t)(t - t_base) * STAGE_PITCH + 4 * ng);
+              u[j] = *reinterpret_cast<const float4 *>(stg + (size_t)(t - t_base) * STAGE_PITCH + 64 + 4 * ng);
             }
           }
         } else {
@@ -595,8 +648,8 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_tc_kernel(const __grid_consta
             const float r = rs[t];
             g[j].x *= r; g[j].y *= r; g[j].z *= r; g[j].w *= r;
             u[j].x *= r; u[j].y *= r; u[j].z *= r; u[j].w *= r;
-            __nv_bfloat162 lo = __floats2bfloat162_rn(g[j].x / (1.0f + __expf(-g[j].x)) * u[j].x, g[j].y / (1.0f + __expf(-g[j].y)) * u[j].y);
-            __nv_bfloat162 hi = __floats2bfloat162_rn(g[j].z / (1.0f + __expf(-g[j].z)) * u[j].z, g[j].w / (1.0f + __expf(-g[j].w)) * u[j].w);
+            __nv_bfloat162 lo = __floats2bfloat162_rn(silu(g[j].x) * u[j].x, silu(g[j].y) * u[j].y);
+            __nv_bfloat162 hi = __floats2bfloat162_rn(silu(g[j].z) * u[j].z, silu(g[j].w) * u[j].w);
             *(uint2 *)(p.out_bf16 + (size_t)t * F + feat) = make_uint2(*(uint32_t *)&lo, *(uint32_t *)&hi);
           }
         }
@@ -611,14 +664,19 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_tc_kernel(const __grid_consta
       bool mine = true;
       if (grp < n_pend) {
         const int tile = pend_tile[grp], n = pend_n[grp], first = pend_first[grp], my = (int)blockIdx.x - first;
-        mine = p.mode == MODE_SWIGLU ? finish_swiglu(tile, gi, 64, grp, my, n, first, nullptr, 0, p.rows)
-                                     : finish_plain(tile, gi, 64, grp, my, n, first, nullptr, 0, p.rows);
+        mine = p.mode == MODE_SWIGLU ? finish_swiglu(tile, gi, 64, grp, my, n, first, nullptr, 0, rows)
+                                     : finish_plain(tile, gi, 64, grp, my, n, first, nullptr, 0, rows);
         if (gi == 0 && grp == 0) TRACE(10);
         if (mine) {
+          if (publish) __threadfence();                                // this thread's outputs, before the tile counts as finished
           group_barrier(grp);
           if (gi == 0) {                                               // the last contributor to finish re-arms the tile
             int d = atomicAdd(p.done + tile, 1);
-            if (d == n - 1) { p.counters[tile] = 0; p.done[tile] = 0; }
+            if (d == n - 1) {
+              p.counters[tile] = 0;
+              p.done[tile] = 0;
+              if (publish) { __threadfence(); atomicAdd(cp.finished + ci, 1); }
+            }
           }
         }
       }
@@ -629,15 +687,24 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_tc_kernel(const __grid_consta
       n_pend = 0;
     };
 
+    if (ci > 0) {
+      // this GEMM's per-token factors are sums over all tiles of the GEMM before it
+      if (et == 0) wait_flag[0] = chain_wait(cp, ci - 1) && !*abort_flag;
+      epi_barrier();
+      ok = wait_flag[0] != 0;
+      epi_barrier();
+      if (!ok) break;
+      __threadfence();
+    }
     if (et < OURO_MAX_ROWS) {
       float r = 1.0f;
-      if (p.ss_in && et < p.rows) {
+      if (p.ss_in && et < rows) {
         float sum = 0.f;
         for (int i = 0; i < p.ss_tiles; ++i) sum += p.ss_in[(size_t)i * OURO_MAX_ROWS + et];
         r = 1.0f / sqrtf(sum * p.ss_inv_d + p.eps);
       }
       rs[et] = r;
-      spos[et] = (p.mode == MODE_QKV && et < p.rows) ? p.pos[et] : 0;
+      spos[et] = (p.mode == MODE_QKV && et < rows) ? p.pos[et] : 0;
     }
     if (et == 0) wait_flag[2] = 0;
     epi_barrier();
@@ -664,7 +731,7 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_tc_kernel(const __grid_consta
           for (int t0 = c0; t0 < c1; t0 += 16) {
             tmem_ld16(taddr + t0, v);
 #pragma unroll
-            for (int i = 0; i < 16; ++i) stage[(t0 - c0 + i) * TILE_N + nl] = v[i];
+            for (int i = 0; i < 16; ++i) stage[(t0 - c0 + i) * STAGE_PITCH + nl] = v[i];
           }
           if (c1 == p.t_pad) {
             fence_before_sync();
@@ -672,10 +739,46 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_tc_kernel(const __grid_consta
             if (lane == 0) mbar_arrive(&acc_empty[a]);
           }
           epi_barrier();
-          const int lim = min(c1, p.rows);
-          if (p.mode == MODE_SWIGLU) finish_swiglu(s.tile, et, 128, 0, 0, 1, 0, stage, c0, lim);
-          else finish_plain(s.tile, et, 128, 0, 0, 1, 0, stage, c0, lim);
+          const int lim = min(c1, rows);
+          if (p.mode == MODE_SWIGLU) {
+            finish_swiglu(s.tile, et, 128, 0, 0, 1, 0, stage, c0, lim);
+          } else if (p.mode == MODE_HEAD) {
+            // greedy choice inside the tile: two threads per token scan 64 parked logits each in ascending index
+            // order (a strict comparison keeps the smallest index among equals), then the halves are compared
+            int seg, row0, col0, valid;
+            locate(p, s.tile, seg, row0, col0, valid);
+            const int t = c0 + (et >> 1), h = et & 1;
+            uint32_t bu = 0;
+            int bi = col0 + 64 * h;
+            if (t < lim) {
+              const float r = rs[t];
+              const float *row = stage + (size_t)(t - c0) * STAGE_PITCH + 64 * h;
+#pragma unroll
+              for (int i = 0; i < 16; ++i) {
+                const float4 x4 = *reinterpret_cast<const float4 *>(row + 4 * i);
+                const float xs[4] = {x4.x * r, x4.y * r, x4.z * r, x4.w * r};
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                  const int cidx = 64 * h + 4 * i + e;
+                  const uint32_t uo = ordered_u32(xs[e]);
+                  if (cidx < valid && uo > bu) { bu = uo; bi = col0 + cidx; }
+                }
+              }
+            }
+            const uint32_t ou = __shfl_xor_sync(0xffffffffu, bu, 1);
+            const int oi = __shfl_xor_sync(0xffffffffu, bi, 1);
+            if (ou > bu || (ou == bu && oi < bi)) { bu = ou; bi = oi; }
+            if (t < lim && h == 0) {
+              p.tile_max[(size_t)s.tile * OURO_MAX_ROWS + t] = ordered_f32(bu);
+              p.tile_arg[(size_t)s.tile * OURO_MAX_ROWS + t] = bi;
+            }
+            if (p.out_f32) finish_plain(s.tile, et, 128, 0, 0, 1, 0, stage, c0, lim);
+          } else {
+            finish_plain(s.tile, et, 128, 0, 0, 1, 0, stage, c0, lim);
+          }
+          if (publish && c1 == p.t_pad) __threadfence();
           epi_barrier();
+          if (publish && c1 == p.t_pad && et == 0) atomicAdd(cp.finished + ci, 1);
         }
       } else {
         // partial tile: park it in this CTA's slot and announce it; the partials are added up after the loop
@@ -684,7 +787,7 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_tc_kernel(const __grid_consta
           tmem_ld16(taddr + t0, v);
 #pragma unroll
           for (int i = 0; i < 16; ++i)
-            if (t0 + i < p.rows) __stcg(mine + (size_t)(t0 + i) * TILE_N + nl, v[i]);
+            if (t0 + i < rows) __stcg(mine + (size_t)(t0 + i) * TILE_N + nl, v[i]);
         }
         fence_before_sync();
         __syncwarp();
@@ -702,7 +805,8 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_tc_kernel(const __grid_consta
     if (et == 0) TRACE(5);
     if (ok) run_fixups();
     if (et == 0) TRACE(7);
-    if (!ok && et == 0) { *abort_flag = 1; atomicExch(p.status, 1); }
+    }
+    if (!ok && et == 0) { *abort_flag = 1; atomicExch(p0.status, 1); }
   }
   // ------------------------------------------------------------------ teardown
   fence_before_sync();
@@ -750,8 +854,15 @@ struct FastState {
   float *tile_max = nullptr;    // LM head: per-tile best logit and index of every token
   int *tile_arg = nullptr;
   float *ss = nullptr;          // per-tile sums of squares of the residual stream (RMSNorm folded into the GEMMs)
+  int *finished = nullptr;      // [MAX_CHAIN] finished-tile counters of the chained GEMMs (device)
+  int finished_host[MAX_CHAIN] = {0, 0, 0, 0};   // the values those counters have once everything launched so far is done
+  ChainParams chain{};          // GEMMs collected for the next launch
+  int chain_kind[MAX_CHAIN] = {0, 0, 0, 0};
+  bool fuse = true;             // run consecutive GEMMs as one launch
+  bool dirty = false;           // a bounded wait gave up: counters must be cleared before the next launch
 };
 constexpr int MAX_TILES = 4096;
+constexpr int SPARE_BYTES = 2048;          // behind the tile counters: chain counters [0, 64), attention arrival counters [64, 512)
 
 size_t slots_bytes() { return (size_t)MAX_GRID * 2 * SLOT_FLOATS * sizeof(float); }
 size_t tile_best_bytes() { return (size_t)MAX_TILES * OURO_MAX_ROWS * 4; }
@@ -760,7 +871,7 @@ size_t ss_bytes() { return (size_t)MAX_SS_TILES * OURO_MAX_ROWS * sizeof(float);
 
 int stages_for(int t_pad, int smem_max) {
   int stage = A_BYTES + t_pad * BLOCK_K * 2;
-  int fixed = 1024 + 64 * OURO_MAX_ROWS * 4 + 1536;  // alignment slack, exchange buffer, barriers, flags, per-token factors and positions
+  int fixed = 1024 + STAGE_BYTES + 1536;  // alignment slack, parked whole tile, barriers, flags, per-token factors and positions
   int s = (smem_max - fixed) / stage;
   return s > 12 ? 12 : s;
 }
@@ -772,7 +883,7 @@ struct ouro_fast { FastState s; };
 size_t ouro_scratch_bytes(const ouro_model_desc *t, const ouro_model_desc *d) {
   size_t attn = attention_tc_scratch_bytes(*t);
   if (d && attention_tc_scratch_bytes(*d) > attn) attn = attention_tc_scratch_bytes(*d);
-  return slots_bytes() + 2 * MAX_TILES * sizeof(int) + 256 + 2 * tile_best_bytes() + ss_bytes() + attn;
+  return slots_bytes() + 2 * MAX_TILES * sizeof(int) + SPARE_BYTES + 2 * tile_best_bytes() + ss_bytes() + attn;
 }
 
 static bool shape_ok(const ouro_model_desc &d) {
@@ -806,11 +917,16 @@ int ouro_fast_setup(ouro_ctx *c) {
   f->s.smem_max = smem;
   f->s.slots = c->a.scratch;
   f->s.counters = (int *)((char *)c->a.scratch + slots_bytes());
-  f->s.tile_max = (float *)((char *)c->a.scratch + slots_bytes() + 2 * MAX_TILES * sizeof(int) + 256);
+  f->s.finished = f->s.counters + 2 * MAX_TILES;               // inside the spare words behind the tile counters
+  {
+    const char *e = getenv("OURO_FUSE");                       // OURO_FUSE=0: every GEMM is a launch of its own
+    f->s.fuse = !(e && e[0] == '0');
+  }
+  f->s.tile_max = (float *)((char *)c->a.scratch + slots_bytes() + 2 * MAX_TILES * sizeof(int) + SPARE_BYTES);
   f->s.tile_arg = (int *)((char *)f->s.tile_max + tile_best_bytes());
   f->s.ss = (float *)((char *)f->s.tile_arg + tile_best_bytes());
   f->s.attn_part = (float *)((char *)f->s.ss + ss_bytes());
-  if (cudaMemsetAsync(f->s.counters, 0, 2 * MAX_TILES * sizeof(int), c->stream) != cudaSuccess ||
+  if (cudaMemsetAsync(f->s.counters, 0, 2 * MAX_TILES * sizeof(int) + SPARE_BYTES, c->stream) != cudaSuccess ||
       cudaFuncSetAttribute(gemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess ||
       attention_tc_setup() != OURO_OK || attention_tm_setup() != OURO_OK) {
     delete f;
@@ -912,8 +1028,27 @@ static int grid_for(const FastState &s, int tiles, int kb) {
   const long total = (long)tiles * kb;
   return total < s.grid ? (int)total : s.grid;
 }
-static void launch_gemm_tc(ouro_ctx *c, GemmParams &p, const CUtensorMap *xmaps, int K, int rows) {
+// Launches the GEMMs collected so far as one chain.
+static void flush_chain(ouro_ctx *c) {
+  FastState &s = c->fast->s;
+  ChainParams &cp = s.chain;
+  if (cp.n == 0) return;
   OURO_COUNT_LAUNCH();
+  int grid = 1;
+  for (int i = 0; i < cp.n; ++i) grid = std::max(grid, grid_for(s, cp.g[i].tiles, cp.g[i].kb));
+  cp.finished = s.finished;
+  for (int i = 0; i + 1 < cp.n; ++i) cp.target[i] = (s.finished_host[i] += cp.g[i].tiles);
+  const bool per_kind = cp.n == 1 && c->prof_class >= OURO_PROF_QKV && c->prof_class <= OURO_PROF_HEAD;
+  static const int kind_class[5] = {OURO_PROF_QKV, OURO_PROF_WO, OURO_PROF_GATEUP, OURO_PROF_DOWN, OURO_PROF_HEAD};
+  {
+    ProfScope ps(c, per_kind ? kind_class[s.chain_kind[0]] : OURO_PROF_GEMM);
+    launch_pdl(gemm_tc_kernel, grid, THREADS, (size_t)s.smem_max, c->stream, cp);
+  }
+  cp.n = 0;
+}
+
+// Adds a GEMM to the chain under construction; `last` launches the chain (something other than a GEMM follows).
+static void push_gemm(ouro_ctx *c, GemmParams &p, int kind, const CUtensorMap *xmaps, int K, int rows, bool last) {
   FastState &s = c->fast->s;
   p.kb = K / BLOCK_K;
   p.rows = rows;
@@ -924,16 +1059,38 @@ static void launch_gemm_tc(ouro_ctx *c, GemmParams &p, const CUtensorMap *xmaps,
   p.counters = s.counters;
   p.done = s.counters + MAX_TILES;
   p.status = &c->st->status;
-  launch_pdl(gemm_tc_kernel, grid_for(s, p.tiles, p.kb), THREADS, (size_t)s.smem_max, c->stream, p);
+  p.rows_dev = c->cur_rows_dev;
+  p.trace_id = kind;
+  if (s.chain.n > 0 && s.chain.g[0].rows != rows) flush_chain(c);   // cannot happen inside one forward
+  s.chain_kind[s.chain.n] = kind;
+  s.chain.g[s.chain.n++] = p;
+  // one launch per GEMM when asked for, and while a single kind of GEMM is being timed
+  const bool split = !s.fuse || (c->prof_class >= OURO_PROF_QKV && c->prof_class <= OURO_PROF_HEAD);
+  if (last || split || s.chain.n == MAX_CHAIN) flush_chain(c);
+}
+
+// Clears what an aborted launch may have left behind (tile counters, chain counters).
+void ouro_fast_reset(ouro_ctx *c, bool force) {
+  if (!c->fast) return;
+  FastState &s = c->fast->s;
+  s.chain.n = 0;
+  if (!force && !s.dirty) return;
+  cudaMemsetAsync(s.counters, 0, 2 * MAX_TILES * sizeof(int) + SPARE_BYTES, c->stream);
+  for (int &v : s.finished_host) v = 0;
+  s.dirty = false;
+}
+void ouro_fast_mark_dirty(ouro_ctx *c) {
+  if (c->fast) c->fast->s.dirty = true;
 }
 
 // Embedding rows into the residual stream, plus what the first norm's consumer needs: bf16(gain * x) and each
 // row's sum of squares (kept in tile 0 of the per-tile array, the other tiles zero).
 __global__ void embed_norm_kernel(const __nv_bfloat16 *E, const int32_t *tok, int d, const __nv_bfloat16 *gain, float *x,
-                                  __nv_bfloat16 *xb, float *ss, int ss_tiles) {
+                                  __nv_bfloat16 *xb, float *ss, int ss_tiles, const int *rows_dev) {
   pdl_trigger();
   pdl_wait();
   const int r = blockIdx.x;
+  if (rows_dev && r >= *rows_dev) return;          // the launch was sized for the largest possible block
   const __nv_bfloat16 *src = E + (size_t)tok[r] * d;
   float sq = 0.f;
   for (int i = threadIdx.x; i < d; i += blockDim.x) {
@@ -955,14 +1112,24 @@ __global__ void embed_norm_kernel(const __nv_bfloat16 *E, const int32_t *tok, in
   for (int i = 1 + threadIdx.x; i < ss_tiles; i += blockDim.x) ss[(size_t)i * OURO_MAX_ROWS + r] = 0.f;
 }
 
+// The row count of a candidate block may stay on the device when every kernel of the forward reads it from there:
+// the tensor-core GEMMs with the rotary epilogue and one of the two tensor-core attention kernels.
+bool ouro_fast_available(ouro_ctx *c, int which) {
+  if (!c->fast || !c->fast->s.m[which].ok) return false;
+  const ouro_model_desc &d = c->m[which].d;
+  return d.head_dim == 64 || d.head_dim == 128;
+}
+
 int ouro_fast_embed(ouro_ctx *c, int which, int rows) {
   if (!c->fast || !c->fast->s.m[which].ok) return OURO_ESTATE;
   ModelRt &M = c->m[which];
   const ouro_model_desc &d = M.d;
+  c->fast->s.chain.n = 0;
   ProfScope ps(c, OURO_PROF_EMBED);
   OURO_COUNT_LAUNCH();
   launch_pdl(embed_norm_kernel, rows, 256, 0, c->stream, (const __nv_bfloat16 *)M.embed, (const int32_t *)M.blk.tok, (int)d.d_model,
-             (const __nv_bfloat16 *)M.attn_norm[0], c->a.x, (__nv_bfloat16 *)c->a.xn, c->fast->s.ss, (int)((d.d_model + TILE_N - 1) / TILE_N));
+             (const __nv_bfloat16 *)M.attn_norm[0], c->a.x, (__nv_bfloat16 *)c->a.xn, c->fast->s.ss, (int)((d.d_model + TILE_N - 1) / TILE_N),
+             (const int *)(M.blk_rows_dev ? &c->st->n_rows : nullptr));
   return OURO_OK;
 }
 
@@ -982,10 +1149,8 @@ int ouro_fast_layer(ouro_ctx *c, int which, int l, int rows) {
   auto consume = [&](GemmParams &p) { p.ss_in = ss; p.ss_tiles = ss_tiles; p.ss_inv_d = 1.0f / (float)d.d_model; p.eps = d.rms_eps; };
   auto produce = [&](GemmParams &p, const void *gain) { p.gain = (const __nv_bfloat16 *)gain; p.xb = (__nv_bfloat16 *)a.xn; p.ss_out = ss; };
   {
-    ProfScope ps(c, OURO_PROF_QKV);
     GemmParams p{};
     set_weights(p, weight_side(d, fm, l, G_QKV));
-    p.trace_id = G_QKV;
     consume(p);
     const bool fused_rope = d.head_dim == 64 || d.head_dim == 128;   // tiles then hold whole heads
     if (fused_rope) {
@@ -1001,7 +1166,7 @@ int ouro_fast_layer(ouro_ctx *c, int which, int l, int rows) {
       p.out_f32 = a.qkv;
       p.ldo = dq + 2 * dkv;
     }
-    launch_gemm_tc(c, p, fm.x_d, d.d_model, rows);
+    push_gemm(c, p, G_QKV, fm.x_d, d.d_model, rows, true);       // closes the chain the previous layer began
     if (!fused_rope) {
       ProfScope pr(c, OURO_PROF_ROPE);
       launch_rope_append(d, a.qkv, M.blk.pos, M.rope_cos, M.rope_sin, rows, M.L, l, a.q, M.k_cache, M.v_cache, s);
@@ -1010,45 +1175,39 @@ int ouro_fast_layer(ouro_ctx *c, int which, int l, int rows) {
   {
     ProfScope ps(c, OURO_PROF_ATTENTION);
     if (c->fast->s.m[which].kv_maps) {
-      if (launch_attention_tm(d, a.q, &c->fast->s.m[which].kmap, &c->fast->s.m[which].vmap, M.k_cache, M.v_cache, M.blk, rows,
-                              M.L, M.L + rows, l, c->fast->s.attn_part, a.att, &c->st->status, s))
-        launch_attention_merge(d, M.blk, rows, c->fast->s.attn_part, a.att, s);
+      launch_attention_tm(d, a.q, &c->fast->s.m[which].kmap, &c->fast->s.m[which].vmap, M.k_cache, M.v_cache, M.blk, rows,
+                          M.L, M.L + rows, l, c->fast->s.attn_part, a.att, &c->st->status, c->fast->s.finished + 64,
+                          c->cur_rows_dev, s);
     } else if (attention_tc_supported(d))
-      launch_attention_tc(d, a.q, M.k_cache, M.v_cache, M.blk, rows, M.L, M.L + rows, l, c->fast->s.attn_part, a.att, s);
+      launch_attention_tc(d, a.q, M.k_cache, M.v_cache, M.blk, rows, M.L, M.L + rows, l, c->fast->s.attn_part, a.att, c->cur_rows_dev, s);
     else
       launch_attention_simple(d, a.q, M.k_cache, M.v_cache, M.blk, rows, l, a.att, s);
   }
   {
-    ProfScope ps(c, OURO_PROF_WO);
     GemmParams p{};
     set_weights(p, weight_side(d, fm, l, G_WO));
-    p.trace_id = G_WO;
     p.mode = MODE_RESIDUAL;
     p.out_f32 = a.x;
     p.ldo = d.d_model;
     produce(p, M.ffn_norm[l]);
-    launch_gemm_tc(c, p, fm.x_q, dq, rows);
+    push_gemm(c, p, G_WO, fm.x_q, dq, rows, false);
   }
   {
-    ProfScope ps(c, OURO_PROF_GATEUP);
     GemmParams p{};
     set_weights(p, weight_side(d, fm, l, G_GATEUP));
-    p.trace_id = G_GATEUP;
     p.mode = MODE_SWIGLU;
     p.out_bf16 = (__nv_bfloat16 *)a.act;
     consume(p);
-    launch_gemm_tc(c, p, fm.x_d, d.d_model, rows);
+    push_gemm(c, p, G_GATEUP, fm.x_d, d.d_model, rows, false);
   }
   {
-    ProfScope ps(c, OURO_PROF_DOWN);
     GemmParams p{};
     set_weights(p, weight_side(d, fm, l, G_DOWN));
-    p.trace_id = G_DOWN;
     p.mode = MODE_RESIDUAL;
     p.out_f32 = a.x;
     p.ldo = d.d_model;
     produce(p, l + 1 < d.n_layers ? M.attn_norm[l + 1] : M.final_norm);
-    launch_gemm_tc(c, p, fm.x_f, d.d_ffn, rows);
+    push_gemm(c, p, G_DOWN, fm.x_f, d.d_ffn, rows, false);     // the next layer's q,k,v or the LM head completes the chain
   }
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) {
@@ -1064,18 +1223,20 @@ __global__ void argmax_tiles_kernel(const float *tile_max, const int *tile_arg, 
   pdl_trigger();
   pdl_wait();
   const int t = blockIdx.x;
-  float bv = -INFINITY;
+  // compared through the same order-preserving integer image as inside the tiles (-0.0 below +0.0), so that the
+  // choice does not depend on where a tile boundary falls
+  uint32_t bv = 0;
   int bi = INT_MAX;
   for (int i = threadIdx.x; i < tiles; i += blockDim.x) {
-    float v = tile_max[(size_t)i * OURO_MAX_ROWS + t];
+    uint32_t v = ordered_u32(tile_max[(size_t)i * OURO_MAX_ROWS + t]);
     int a = tile_arg[(size_t)i * OURO_MAX_ROWS + t];
     if (v > bv || (v == bv && a < bi)) { bv = v; bi = a; }
   }
-  __shared__ float sv[8];
+  __shared__ uint32_t sv[8];
   __shared__ int si[8];
 #pragma unroll
   for (int o = 16; o; o >>= 1) {
-    float ov = __shfl_xor_sync(0xffffffffu, bv, o);
+    uint32_t ov = __shfl_xor_sync(0xffffffffu, bv, o);
     int oi = __shfl_xor_sync(0xffffffffu, bi, o);
     if (ov > bv || (ov == bv && oi < bi)) { bv = ov; bi = oi; }
   }
@@ -1094,17 +1255,15 @@ int ouro_fast_head(ouro_ctx *c, int which, int rows, float *logits, int32_t *arg
   FastModel &fm = c->fast->s.m[which];
   const ouro_model_desc &d = M.d;
   {
-    ProfScope ps(c, OURO_PROF_HEAD);
     GemmParams p{};
     set_weights(p, weight_side(d, fm, 0, G_HEAD));
-    p.trace_id = G_HEAD;
     p.mode = MODE_HEAD;
     p.out_f32 = logits;
     p.ldo = d.vocab;
     p.tile_max = c->fast->s.tile_max;
     p.tile_arg = c->fast->s.tile_arg;
     p.ss_in = c->fast->s.ss; p.ss_tiles = (d.d_model + TILE_N - 1) / TILE_N; p.ss_inv_d = 1.0f / (float)d.d_model; p.eps = d.rms_eps;
-    launch_gemm_tc(c, p, fm.x_d, d.d_model, rows);
+    push_gemm(c, p, G_HEAD, fm.x_d, d.d_model, rows, true);
   }
   {
     ProfScope ps(c, OURO_PROF_ARGMAX);
@@ -1207,7 +1366,9 @@ extern "C" int ouro_lm_head_static(const void *x_dev, const void *lm_head_dev, i
   const int tiles = (vocab + TILE_N - 1) / TILE_N;
   // the array keeps whatever the last call left: counters and status must start at zero
   cudaError_t e = cudaMemsetAsync(base + NA_OFF_COUNTERS, 0, NA_OFF_TMAX - NA_OFF_COUNTERS, s);
-  GemmParams p{};
+  ChainParams cp{};
+  cp.n = 1;
+  GemmParams &p = cp.g[0];
   const int t_pad = (rows + 15) & ~15;
   if (e != cudaSuccess || !make_map(&p.a[0], lm_head_dev, vocab, d_model, TILE_N) || !make_map(&p.b, x_dev, rows, d_model, t_pad)) {
     ouro_set_global_error("ouro_lm_head_static: could not describe the operands to the copy engine");
@@ -1229,7 +1390,7 @@ extern "C" int ouro_lm_head_static(const void *x_dev, const void *lm_head_dev, i
   p.done = p.counters + NA_MAX_TILES;
   p.status = (int *)(base + NA_OFF_STATUS);
   const int total = tiles * p.kb;
-  gemm_tc_kernel<<<total < NA_GRID ? total : NA_GRID, THREADS, g_na_smem[dev], s>>>(p);
+  gemm_tc_kernel<<<total < NA_GRID ? total : NA_GRID, THREADS, g_na_smem[dev], s>>>(cp);
   argmax_tiles_kernel<<<rows, 128, 0, s>>>(p.tile_max, p.tile_arg, tiles, argmax_dev);
   int status = 0;
   if ((e = cudaGetLastError()) != cudaSuccess ||

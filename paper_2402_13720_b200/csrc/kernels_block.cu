@@ -278,6 +278,7 @@ __device__ void accept_body(const BlockDev &b, DevState *st, const int32_t *o, i
     for (int i = 0; i < m; ++i) st->accepted[n++] = b.tok[1 + gamma + chosen * S + i];
   }
   st->accepted[n++] = bonus;
+  st->n_cand_last = nc;
   st->A = A;
   st->chosen = chosen;
   st->m = m;
@@ -392,7 +393,7 @@ __global__ void accept_compact_harvest_kernel(BlockDev b, DevState *st, PoolDev 
   if (blockIdx.x == 0) {
     if (threadIdx.x == 0) {
       accept_body(b, st, o, seq_dev, gamma, S);
-      if (mbox) mbox_post(mbox + MBOX_ACCEPT, &st->A, 4 + OURO_MAX_GAMMA + OURO_MAX_BETA + 1, seq);   // A .. status
+      if (mbox) mbox_post(mbox + MBOX_ACCEPT, &st->A, 4 + OURO_MAX_GAMMA + OURO_MAX_BETA + 2, seq);   // A .. n_cand_last
     }
     __syncthreads();
     if (threadIdx.x < 32 && (flags & (OURO_HARVEST_MATCHED | OURO_HARVEST_CANDIDATES | OURO_HARVEST_ACCEPTED)))

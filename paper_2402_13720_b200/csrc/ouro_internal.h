@@ -51,7 +51,7 @@ struct DevState {
   int32_t n_acc;     // tokens accepted by the last verification
   int32_t accepted[OURO_MAX_GAMMA + OURO_MAX_BETA];
   int32_t status;    // sticky device-side error word (0 = fine)
-  int32_t pad;
+  int32_t n_cand_last;  // copy of n_cand taken at acceptance (the acceptance record A .. n_cand_last is read back as one piece)
   u64 clock;         // phrase-pool stamp counter
   // last phrase-level drafting round of the draft model (Section 3.1)
   int32_t d_keep;    // draft tokens the round added (at most what was still missing of gamma)
@@ -86,6 +86,7 @@ struct ModelRt {
   int32_t blk_rows = 0; // rows of the current block (0 = none assembled)
   int32_t blk_L = -1;   // cache length the block was assembled for
   bool blk_is_candidate = false;
+  bool blk_rows_dev = false;  // blk_rows is an upper bound; the true count is DevState::n_rows (tensor-core path only)
 };
 
 struct Activations {  // sized for OURO_MAX_ROWS rows of the larger model
@@ -123,6 +124,7 @@ struct ouro_ctx {
   // record) are written there by the kernels themselves, payload first, then a sequence number the host polls.
   int32_t *mbox = nullptr, *mbox_dev = nullptr;
   int32_t mseq = 0;
+  const int *cur_rows_dev = nullptr;   // during a forward: where the kernels read the block's true row count, or NULL
   ouro_drafter_fn drafter = nullptr;
   void *drafter_user = nullptr;
   int32_t step = 0;
@@ -200,12 +202,13 @@ bool attention_tc_supported(const ouro_model_desc &d);
 size_t attention_tc_scratch_bytes(const ouro_model_desc &d);
 int attention_tc_setup();
 void launch_attention_tc(const ouro_model_desc &d, const void *q, const void *k_cache, const void *v_cache, const BlockDev &b,
-                         int rows, int L, int n_vis_max, int layer, float *part, void *out, cudaStream_t s);
-void launch_attention_merge(const ouro_model_desc &d, const BlockDev &b, int rows, float *part, void *out, cudaStream_t s);
+                         int rows, int L, int n_vis_max, int layer, float *part, void *out, const int *rows_dev, cudaStream_t s);
+void launch_attention_merge(const ouro_model_desc &d, const BlockDev &b, int rows, float *part, void *out, const int *rows_dev,
+                            cudaStream_t s);
 
 // ---- attn_tm.cu (tcgen05 path, head dim 128) ---------------------------------------------------
 bool attention_tm_supported(const ouro_model_desc &d);
 int attention_tm_setup();
-bool launch_attention_tm(const ouro_model_desc &d, const void *q, const void *kmap, const void *vmap, const void *k_cache,
+void launch_attention_tm(const ouro_model_desc &d, const void *q, const void *kmap, const void *vmap, const void *k_cache,
                          const void *v_cache, const BlockDev &b, int rows, int L, int n_vis_max, int layer, float *part,
-                         void *out, int *status, cudaStream_t s);
+                         void *out, int *status, int *arrived, const int *rows_dev, cudaStream_t s);

@@ -71,11 +71,11 @@ def main():
     spans = []
     for kind in range(5):
         t = g[kind]
-        live = t[:, 0] > 0
+        live = t[:, 1] > 0                       # stamped by every GEMM of a chained launch (slot 0: by its first only)
         if not live.any():
             continue
         t = t[live]
-        t0 = t[:, 1][t[:, 1] > 0].min()
+        t0 = t[:, 1].min()
         print(f"{names[kind]}  ({live.sum()} CTAs; us relative to the end of the dependency wait)")
         for col, nm in points:
             x = t[:, col][t[:, col] > 0]
