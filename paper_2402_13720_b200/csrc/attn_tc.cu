@@ -395,43 +395,11 @@ __global__ void __launch_bounds__(THREADS) attn_span_kernel(const AttnParams p) 
   }
 }
 
-// Folds a row's spans and normalises.  One warp per (row, head).  First the largest span maximum, then one
-// weighted sum over the spans in ascending order: the loads of different spans do not wait for one another.
-template <int HD>
-__global__ void attn_merge_kernel(const AttnParams p) {
-  constexpr int PW = HD + 2, DPL = HD / 32;
-  pdl_trigger();
-  pdl_wait();
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int r = blockIdx.x, head = blockIdx.y * (blockDim.x >> 5) + warp;
-  if (head >= p.H || (p.rows_dev && r >= __ldg(p.rows_dev))) return;
-  const int nv = p.lin_end[r] + p.seg_len[r];
-  const int ns = (nv + SPAN - 1) / SPAN;
-  const float *src = p.part + ((size_t)r * p.H + head) * p.cap * PW;
-  float mx = -INFINITY;
-  for (int c = lane; c < ns; c += 32) mx = fmaxf(mx, src[(size_t)c * PW]);
-#pragma unroll
-  for (int o = 16; o; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
-  float l = 0.f, acc[DPL];
-#pragma unroll
-  for (int i = 0; i < DPL; ++i) acc[i] = 0.f;
-#pragma unroll 4
-  for (int c = 0; c < ns; ++c) {
-    const float *pc = src + (size_t)c * PW;
-    const float mp = pc[0];
-    const float w = (mp == -INFINITY) ? 0.f : exp2f(mp - mx);     // mx is finite: the first span holds a visible key
-    l += pc[1] * w;
-#pragma unroll
-    for (int i = 0; i < DPL; ++i) acc[i] += pc[2 + lane + 32 * i] * w;
-  }
-  const float inv = 1.0f / l;
-#pragma unroll
-  for (int i = 0; i < DPL; ++i) p.out[(size_t)r * p.H * HD + head * HD + lane + 32 * i] = __float2bfloat16_rn(acc[i] * inv);
-}
-
 }  // namespace
 
-bool attention_tc_supported(const ouro_model_desc &d) { return d.dtype == OURO_BF16 && (d.head_dim == 64 || d.head_dim == 128); }
+bool attention_tc_supported(const ouro_model_desc &d) {
+  return d.dtype == OURO_BF16 && (d.head_dim == 64 || d.head_dim == 128) && d.max_seq <= 32 * SPAN;   // the fold looks at one span per lane
+}
 
 size_t attention_tc_scratch_bytes(const ouro_model_desc &d) {
   if (!attention_tc_supported(d)) return 0;
@@ -447,26 +415,8 @@ int attention_tc_setup() {
   return OURO_OK;
 }
 
-// Folds the per-span pieces written by either span kernel (head dim 64 or 128) into the block's attention output.
-void launch_attention_merge(const ouro_model_desc &d, const BlockDev &b, int rows, float *part, void *out, const int *rows_dev,
-                            cudaStream_t s) {
-  OURO_COUNT_LAUNCH();
-  AttnParams p{};
-  p.rows_dev = rows_dev;
-  p.lin_end = b.lin_end; p.seg_start = b.seg_start; p.seg_len = b.seg_len; p.group = b.group;
-  p.rows = rows; p.H = d.n_heads; p.Hkv = d.n_kv_heads;
-  p.cap = (d.max_seq + SPAN - 1) / SPAN;
-  p.part = part;
-  p.out = (__nv_bfloat16 *)out;
-  dim3 mgrid(rows, (d.n_heads + 3) / 4);
-  if (d.head_dim == 128)
-    launch_pdl(attn_merge_kernel<128>, mgrid, 128, 0, s, p);
-  else
-    launch_pdl(attn_merge_kernel<64>, mgrid, 128, 0, s, p);
-}
-
 // n_vis_max: an upper bound of the number of keys any row of the block sees (cache length + rows).
-void launch_attention_tc(const ouro_model_desc &d, const void *q, const void *k_cache, const void *v_cache, const BlockDev &b,
+bool launch_attention_tc(const ouro_model_desc &d, const void *q, const void *k_cache, const void *v_cache, const BlockDev &b,
                          int rows, int L, int n_vis_max, int layer, float *part, void *out, const int *rows_dev, cudaStream_t s) {
   OURO_COUNT_LAUNCH();
   AttnParams p;
@@ -482,14 +432,9 @@ void launch_attention_tc(const ouro_model_desc &d, const void *q, const void *k_
   p.part = part;
   p.out = (__nv_bfloat16 *)out;
   const int m_all = (d.n_heads / d.n_kv_heads) * rows;      // query rows per kv head, served 64 per CTA
-  dim3 grid((n_vis_max + SPAN - 1) / SPAN, d.n_kv_heads, (m_all + QR - 1) / QR), mgrid(rows, (d.n_heads + 3) / 4);
-  p.direct = n_vis_max <= SPAN;                             // a single span: nothing to fold, no second launch
-  if (!p.direct) OURO_COUNT_LAUNCH();
-  if (d.head_dim == 128) {
-    launch_pdl(attn_span_kernel<128>, grid, THREADS, Smem<128>::BYTES, s, p);
-    if (!p.direct) launch_pdl(attn_merge_kernel<128>, mgrid, 128, 0, s, p);
-  } else {
-    launch_pdl(attn_span_kernel<64>, grid, THREADS, Smem<64>::BYTES, s, p);
-    if (!p.direct) launch_pdl(attn_merge_kernel<64>, mgrid, 128, 0, s, p);
-  }
+  dim3 grid((n_vis_max + SPAN - 1) / SPAN, d.n_kv_heads, (m_all + QR - 1) / QR);
+  p.direct = n_vis_max <= SPAN;                             // a single span: nothing to fold
+  if (d.head_dim == 128) launch_pdl(attn_span_kernel<128>, grid, THREADS, Smem<128>::BYTES, s, p);
+  else launch_pdl(attn_span_kernel<64>, grid, THREADS, Smem<64>::BYTES, s, p);
+  return !p.direct;
 }

@@ -99,7 +99,6 @@ struct TmParams {
   int direct;                      // every row's keys lie in span 0: normalise and write `out`, no folding needed
   int *status;
   const int *rows_dev;             // NULL, or the block's true row count in device memory (`rows` is then an upper bound)
-  int *arrived;                    // [Hkv * rounds] CTAs of a (kv head, round) that have written their span; zero between launches
 };
 
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -625,7 +624,6 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tm_kernel(const __grid_consta
       }
     }
   }
-  if (!p.direct) __threadfence();                       // this thread's span pieces, before the CTA counts as arrived
   fence_before_sync();
   __syncthreads();
   if (tid == 0) TRACE(5);
@@ -633,83 +631,12 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tm_kernel(const __grid_consta
     fence_after_sync();
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(512u));
   }
-  if (p.direct) return;
-  // ---- folding the spans: the CTA that arrives last for its (kv head, round) has every span's piece in front of it
-  //      and folds them for the round's query rows - first the largest span maximum, then one weighted sum over the
-  //      spans in ascending order, one warp per (row, head).  The arithmetic of a row involves its own spans only.
-  if (tid == 0) {
-    int *cnt = p.arrived + blockIdx.y * p.Hkv + kvh;
-    const int prev = atomicAdd(cnt, 1);
-    ms->n_items = prev == p.n_spans - 1;                // reused as the "I am last" flag
-    if (prev == p.n_spans - 1) *cnt = 0;                // ready for the next launch
-  }
-  __syncthreads();
-  if (!ms->n_items) return;
-  __threadfence();
-  // Two (row, head) pairs per warp and pass, so that their loads overlap; per pair: lane c fetches span c's maximum
-  // and sum (at most 32 spans), then every lane fetches its four dims of every span before the first is used.
-  constexpr int NW = THREADS / 32, UNR = 12;
-  for (int t0 = warp; t0 < QR; t0 += 2 * NW) {
-    const float *src[2];
-    int ns[2], oidx[2];
-    float m_l[2], l_l[2];
-#pragma unroll
-    for (int k = 0; k < 2; ++k) {
-      const int t = t0 + k * NW, info = t < QR ? ms->map[t] : -1;
-      ns[k] = 0;
-      src[k] = p.part;
-      oidx[k] = 0;
-      if (info >= 0) {
-        const int r = info & 0xff, head = kvh * g + ((info >> 8) & 0xff);
-        ns[k] = (ms->lin[r] + ms->len[r] + SPAN - 1) / SPAN;
-        src[k] = p.part + ((size_t)r * p.H + head) * p.cap * PW;
-        oidx[k] = (r * p.H + head) * HD;
-      }
-      m_l[k] = -INFINITY;
-      l_l[k] = 0.f;
-      if (lane < ns[k]) {
-        m_l[k] = __ldcg(src[k] + (size_t)lane * PW);
-        l_l[k] = __ldcg(src[k] + (size_t)lane * PW + 1);
-      }
-    }
-#pragma unroll
-    for (int k = 0; k < 2; ++k) {
-      if (ns[k] == 0) continue;                                    // uniform in the warp
-      float mx = m_l[k];
-#pragma unroll
-      for (int o = 16; o; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
-      const float w_l = (m_l[k] == -INFINITY) ? 0.f : exp2f(m_l[k] - mx);   // mx is finite: the first span holds a visible key
-      float l = 0.f, acc[HD / 32];
-#pragma unroll
-      for (int i = 0; i < HD / 32; ++i) acc[i] = 0.f;
-      for (int c0 = 0; c0 < ns[k]; c0 += UNR) {
-        float o[UNR][HD / 32];
-#pragma unroll
-        for (int cc = 0; cc < UNR; ++cc)
-#pragma unroll
-          for (int i = 0; i < HD / 32; ++i)
-            o[cc][i] = c0 + cc < ns[k] ? __ldcg(src[k] + (size_t)(c0 + cc) * PW + 2 + lane + 32 * i) : 0.f;
-#pragma unroll
-        for (int cc = 0; cc < UNR; ++cc) {
-          if (c0 + cc >= ns[k]) break;                              // uniform in the warp
-          const float w = __shfl_sync(0xffffffffu, w_l, c0 + cc);
-          l += __shfl_sync(0xffffffffu, l_l[k], c0 + cc) * w;
-#pragma unroll
-          for (int i = 0; i < HD / 32; ++i) acc[i] += o[cc][i] * w;
-        }
-      }
-      const float inv = 1.0f / l;
-#pragma unroll
-      for (int i = 0; i < HD / 32; ++i) p.out[(size_t)oidx[k] + lane + 32 * i] = __float2bfloat16_rn(acc[i] * inv);
-    }
-  }
 }
 
 }  // namespace
 
 bool attention_tm_supported(const ouro_model_desc &d) {
   return d.dtype == OURO_BF16 && d.head_dim == HD && d.n_heads % d.n_kv_heads == 0 && d.n_heads / d.n_kv_heads <= 255 &&
-         d.n_heads + d.n_kv_heads <= 448 &&   // arrival counters: one per (kv head, round of 128 query rows)
          d.max_seq <= 32 * SPAN;              // the fold looks at one span per lane
 }
 
@@ -719,11 +646,11 @@ int attention_tm_setup() {
 }
 
 // kmap / vmap: CUtensorMap objects over the whole K and V caches, [n_layers * max_seq][Hkv * 128] bf16 with a
-// 64 x 128 box in 128-byte swizzle.  One launch: the spans are folded by the kernel itself.  `arrived` points at
-// Hkv * rounds zeroed ints that the kernel leaves zeroed.
-void launch_attention_tm(const ouro_model_desc &d, const void *q, const void *kmap, const void *vmap, const void *k_cache,
+// 64 x 128 box in 128-byte swizzle.  Returns true when the spans still have to be folded (attn_fold.cuh: by the kernel
+// that consumes the attention output); with a single span the kernel has written `out` itself.
+bool launch_attention_tm(const ouro_model_desc &d, const void *q, const void *kmap, const void *vmap, const void *k_cache,
                          const void *v_cache, const BlockDev &b, int rows, int L, int n_vis_max, int layer, float *part,
-                         void *out, int *status, int *arrived, const int *rows_dev, cudaStream_t s) {
+                         void *out, int *status, const int *rows_dev, cudaStream_t s) {
   OURO_COUNT_LAUNCH();
   TmParams p;
   p.kmap = *reinterpret_cast<const CUtensorMap *>(kmap);
@@ -741,10 +668,10 @@ void launch_attention_tm(const ouro_model_desc &d, const void *q, const void *km
   p.out = (__nv_bfloat16 *)out;
   p.direct = n_vis_max <= SPAN;
   p.status = status;
-  p.arrived = arrived;
   p.rows_dev = rows_dev;
   const int m_all = (d.n_heads / d.n_kv_heads) * rows;
   p.n_spans = (n_vis_max + SPAN - 1) / SPAN;
   dim3 grid(p.n_spans * d.n_kv_heads, (m_all + QR - 1) / QR);
   launch_pdl(attn_tm_kernel, grid, THREADS, SMEM_BYTES, s, p);
+  return !p.direct;
 }

@@ -23,6 +23,7 @@
 
 #include "ouro_internal.h"
 #include "weight_stream.cuh"
+#include "attn_fold.cuh"
 
 void ouro_set_global_error(const std::string &msg);   // api.cu
 
@@ -110,8 +111,12 @@ constexpr int MAX_CHAIN = 4;
 struct ChainParams {
   GemmParams g[MAX_CHAIN];
   int n;
-  int *finished;            // [MAX_CHAIN] tiles finished, per chain position (monotonic)
+  int *finished;            // [MAX_CHAIN + 1] tiles finished, per chain position (monotonic); last: CTAs done folding
   int target[MAX_CHAIN];    // value finished[i] has when GEMM i of this launch is complete
+  // The first GEMM's activations may be the attention output, still in per-span pieces: every CTA first folds a share
+  // of the (row, head) pairs, and the first activation tile is fetched once all CTAs have.
+  fold::Params fold;
+  int fold_target;
 };
 static_assert(sizeof(ChainParams) <= 4096, "kernel parameters");
 
@@ -311,6 +316,15 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_tc_kernel(const __grid_consta
       pdl_wait();                                  // the first GEMM's activations are the previous kernel's output
       uint32_t n = 0;
       bool ok = true;
+      if (cp.fold.part) {                          // ... once every CTA has folded its share of the attention spans
+        ok = false;
+        for (uint32_t spin = 0; spin < (1u << 22) && !ok; ++spin) {
+          int seen;
+          asm volatile("ld.acquire.gpu.global.b32 %0, [%1];" : "=r"(seen) : "l"(cp.finished + MAX_CHAIN) : "memory");
+          ok = seen - cp.fold_target >= 0;
+        }
+        asm volatile("fence.proxy.async;" ::: "memory");
+      }
       for (int ci = 0; ci < cp.n && ok; ++ci) {
         const GemmParams &p = cp.g[ci];
         if (ci > 0) {
@@ -381,6 +395,12 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_tc_kernel(const __grid_consta
     uint32_t item = 0;
     bool ok = true;
     float v[16];
+    if (cp.fold.part) {
+      fold::run(cp.fold, (int)blockIdx.x * 4 + (warp - 2), (int)gridDim.x * 4, lane);
+      __threadfence();
+      epi_barrier();
+      if (et == 0) atomicAdd(cp.finished + MAX_CHAIN, 1);
+    }
     for (int ci = 0; ci < cp.n && ok; ++ci) {
     const GemmParams &p = cp.g[ci];
     const bool publish = ci + 1 < cp.n;          // a later GEMM of the chain consumes this one's output
@@ -855,7 +875,7 @@ struct FastState {
   int *tile_arg = nullptr;
   float *ss = nullptr;          // per-tile sums of squares of the residual stream (RMSNorm folded into the GEMMs)
   int *finished = nullptr;      // [MAX_CHAIN] finished-tile counters of the chained GEMMs (device)
-  int finished_host[MAX_CHAIN] = {0, 0, 0, 0};   // the values those counters have once everything launched so far is done
+  int finished_host[MAX_CHAIN + 1] = {0, 0, 0, 0, 0};   // the values those counters have once everything launched so far is done
   ChainParams chain{};          // GEMMs collected for the next launch
   int chain_kind[MAX_CHAIN] = {0, 0, 0, 0};
   bool fuse = true;             // run consecutive GEMMs as one launch
@@ -1038,6 +1058,7 @@ static void flush_chain(ouro_ctx *c) {
   for (int i = 0; i < cp.n; ++i) grid = std::max(grid, grid_for(s, cp.g[i].tiles, cp.g[i].kb));
   cp.finished = s.finished;
   for (int i = 0; i + 1 < cp.n; ++i) cp.target[i] = (s.finished_host[i] += cp.g[i].tiles);
+  if (cp.fold.part) cp.fold_target = (s.finished_host[MAX_CHAIN] += grid);
   const bool per_kind = cp.n == 1 && c->prof_class >= OURO_PROF_QKV && c->prof_class <= OURO_PROF_HEAD;
   static const int kind_class[5] = {OURO_PROF_QKV, OURO_PROF_WO, OURO_PROF_GATEUP, OURO_PROF_DOWN, OURO_PROF_HEAD};
   {
@@ -1045,6 +1066,7 @@ static void flush_chain(ouro_ctx *c) {
     launch_pdl(gemm_tc_kernel, grid, THREADS, (size_t)s.smem_max, c->stream, cp);
   }
   cp.n = 0;
+  cp.fold.part = nullptr;
 }
 
 // Adds a GEMM to the chain under construction; `last` launches the chain (something other than a GEMM follows).
@@ -1074,6 +1096,7 @@ void ouro_fast_reset(ouro_ctx *c, bool force) {
   if (!c->fast) return;
   FastState &s = c->fast->s;
   s.chain.n = 0;
+  s.chain.fold.part = nullptr;
   if (!force && !s.dirty) return;
   cudaMemsetAsync(s.counters, 0, 2 * MAX_TILES * sizeof(int) + SPARE_BYTES, c->stream);
   for (int &v : s.finished_host) v = 0;
@@ -1125,6 +1148,7 @@ int ouro_fast_embed(ouro_ctx *c, int which, int rows) {
   ModelRt &M = c->m[which];
   const ouro_model_desc &d = M.d;
   c->fast->s.chain.n = 0;
+  c->fast->s.chain.fold.part = nullptr;
   ProfScope ps(c, OURO_PROF_EMBED);
   OURO_COUNT_LAUNCH();
   launch_pdl(embed_norm_kernel, rows, 256, 0, c->stream, (const __nv_bfloat16 *)M.embed, (const int32_t *)M.blk.tok, (int)d.d_model,
@@ -1174,14 +1198,27 @@ int ouro_fast_layer(ouro_ctx *c, int which, int l, int rows) {
   }
   {
     ProfScope ps(c, OURO_PROF_ATTENTION);
-    if (c->fast->s.m[which].kv_maps) {
-      launch_attention_tm(d, a.q, &c->fast->s.m[which].kmap, &c->fast->s.m[which].vmap, M.k_cache, M.v_cache, M.blk, rows,
-                          M.L, M.L + rows, l, c->fast->s.attn_part, a.att, &c->st->status, c->fast->s.finished + 64,
-                          c->cur_rows_dev, s);
-    } else if (attention_tc_supported(d))
-      launch_attention_tc(d, a.q, M.k_cache, M.v_cache, M.blk, rows, M.L, M.L + rows, l, c->fast->s.attn_part, a.att, c->cur_rows_dev, s);
+    bool pieces = false;             // the attention output is still in per-span pieces
+    if (c->fast->s.m[which].kv_maps)
+      pieces = launch_attention_tm(d, a.q, &c->fast->s.m[which].kmap, &c->fast->s.m[which].vmap, M.k_cache, M.v_cache, M.blk, rows,
+                                   M.L, M.L + rows, l, c->fast->s.attn_part, a.att, &c->st->status, c->cur_rows_dev, s);
+    else if (attention_tc_supported(d))
+      pieces = launch_attention_tc(d, a.q, M.k_cache, M.v_cache, M.blk, rows, M.L, M.L + rows, l, c->fast->s.attn_part, a.att,
+                                   c->cur_rows_dev, s);
     else
       launch_attention_simple(d, a.q, M.k_cache, M.v_cache, M.blk, rows, l, a.att, s);
+    if (pieces) {                    // folded by the output projection's launch, all its CTAs taking part
+      fold::Params &f = c->fast->s.chain.fold;
+      f.part = c->fast->s.attn_part;
+      f.out = (__nv_bfloat16 *)a.att;
+      f.lin_end = M.blk.lin_end;
+      f.seg_len = M.blk.seg_len;
+      f.rows_dev = c->cur_rows_dev;
+      f.rows = rows;
+      f.H = d.n_heads;
+      f.cap = (d.max_seq + fold::SPAN_KEYS - 1) / fold::SPAN_KEYS;
+      f.head_dim = d.head_dim;
+    }
   }
   {
     GemmParams p{};

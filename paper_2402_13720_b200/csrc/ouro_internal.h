@@ -201,14 +201,13 @@ void launch_attention_simple(const ouro_model_desc &d, const void *q, const void
 bool attention_tc_supported(const ouro_model_desc &d);
 size_t attention_tc_scratch_bytes(const ouro_model_desc &d);
 int attention_tc_setup();
-void launch_attention_tc(const ouro_model_desc &d, const void *q, const void *k_cache, const void *v_cache, const BlockDev &b,
+// Both return true when the spans still have to be folded by the kernel that consumes `out` (attn_fold.cuh).
+bool launch_attention_tc(const ouro_model_desc &d, const void *q, const void *k_cache, const void *v_cache, const BlockDev &b,
                          int rows, int L, int n_vis_max, int layer, float *part, void *out, const int *rows_dev, cudaStream_t s);
-void launch_attention_merge(const ouro_model_desc &d, const BlockDev &b, int rows, float *part, void *out, const int *rows_dev,
-                            cudaStream_t s);
 
 // ---- attn_tm.cu (tcgen05 path, head dim 128) ---------------------------------------------------
 bool attention_tm_supported(const ouro_model_desc &d);
 int attention_tm_setup();
-void launch_attention_tm(const ouro_model_desc &d, const void *q, const void *kmap, const void *vmap, const void *k_cache,
+bool launch_attention_tm(const ouro_model_desc &d, const void *q, const void *kmap, const void *vmap, const void *k_cache,
                          const void *v_cache, const BlockDev &b, int rows, int L, int n_vis_max, int layer, float *part,
-                         void *out, int *status, int *arrived, const int *rows_dev, cudaStream_t s);
+                         void *out, int *status, const int *rows_dev, cudaStream_t s);
