@@ -116,7 +116,18 @@ struct ChainParams {
   // The first GEMM's activations may be the attention output, still in per-span pieces: every CTA first folds a share
   // of the (row, head) pairs, and the first activation tile is fetched once all CTAs have.
   fold::Params fold;
-  int fold_target;
+  int fold_target;                // value finished[MAX_CHAIN] has once every CTA has done its share of the work in front
+  // ... or the embedding rows of the block's tokens (first layer): gathered by all CTAs the same way.
+  struct Embed {
+    const __nv_bfloat16 *table;   // [vocab][d]; NULL: nothing to gather
+    const int32_t *tok;           // [rows]
+    const __nv_bfloat16 *gain;    // first norm's gain [d]
+    float *x;                     // residual stream [rows][d]
+    __nv_bfloat16 *xb;            // bf16(gain * x) [rows][d]
+    float *ss;                    // [d / 128][128] sums of squares per 128-column tile
+    const int *rows_dev;
+    int rows, d;
+  } embed;
 };
 static_assert(sizeof(ChainParams) <= 4096, "kernel parameters");
 
@@ -316,7 +327,7 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_tc_kernel(const __grid_consta
       pdl_wait();                                  // the first GEMM's activations are the previous kernel's output
       uint32_t n = 0;
       bool ok = true;
-      if (cp.fold.part) {                          // ... once every CTA has folded its share of the attention spans
+      if (cp.fold.part || cp.embed.table) {        // ... once every CTA has done its share of the fold / the gather
         ok = false;
         for (uint32_t spin = 0; spin < (1u << 22) && !ok; ++spin) {
           int seen;
@@ -395,11 +406,54 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_tc_kernel(const __grid_consta
     uint32_t item = 0;
     bool ok = true;
     float v[16];
-    if (cp.fold.part) {
-      fold::run(cp.fold, (int)blockIdx.x * 4 + (warp - 2), (int)gridDim.x * 4, lane);
+    if (cp.fold.part || cp.embed.table) {
+      const int gw = (int)blockIdx.x * 4 + (warp - 2), nw = (int)gridDim.x * 4;
+      if (cp.fold.part) {
+        fold::run(cp.fold, gw, nw, lane);
+      } else {
+        // Embedding rows into the residual stream, plus what the first norm's consumer needs: bf16(gain * x) and the
+        // sums of squares per 128-column tile.  One warp per (row, tile): four columns per lane.
+        const ChainParams::Embed &e = cp.embed;
+        const int rows = e.rows_dev ? min(e.rows, __ldg(e.rows_dev)) : e.rows, tiles = (e.d + TILE_N - 1) / TILE_N;
+        for (int it = gw; it < rows * tiles; it += nw) {
+          const int r = it / tiles, col = (it - r * tiles) * TILE_N + 4 * lane;
+          float sq = 0.f;
+          if (col < e.d) {                                            // d is a multiple of 64: four columns are in or out together
+            const uint2 raw = __ldg(reinterpret_cast<const uint2 *>(e.table + (size_t)__ldg(e.tok + r) * e.d + col));
+            const uint2 graw = __ldg(reinterpret_cast<const uint2 *>(e.gain + col));
+            const __nv_bfloat162 a01 = *reinterpret_cast<const __nv_bfloat162 *>(&raw.x), a23 = *reinterpret_cast<const __nv_bfloat162 *>(&raw.y);
+            const __nv_bfloat162 g01 = *reinterpret_cast<const __nv_bfloat162 *>(&graw.x), g23 = *reinterpret_cast<const __nv_bfloat162 *>(&graw.y);
+            const float v[4] = {__low2float(a01), __high2float(a01), __low2float(a23), __high2float(a23)};
+            const float gv[4] = {__low2float(g01), __high2float(g01), __low2float(g23), __high2float(g23)};
+            *reinterpret_cast<float4 *>(e.x + (size_t)r * e.d + col) = make_float4(v[0], v[1], v[2], v[3]);
+            __nv_bfloat162 lo = __floats2bfloat162_rn(gv[0] * v[0], gv[1] * v[1]), hi = __floats2bfloat162_rn(gv[2] * v[2], gv[3] * v[3]);
+            *reinterpret_cast<uint2 *>(e.xb + (size_t)r * e.d + col) = make_uint2(*(uint32_t *)&lo, *(uint32_t *)&hi);
+            sq = (v[0] * v[0] + v[1] * v[1]) + (v[2] * v[2] + v[3] * v[3]);
+          }
+#pragma unroll
+          for (int o = 16; o; o >>= 1) sq += __shfl_xor_sync(0xffffffffu, sq, o);
+          if (lane == 0) e.ss[(size_t)(it - r * tiles) * OURO_MAX_ROWS + r] = sq;
+        }
+      }
       __threadfence();
       epi_barrier();
       if (et == 0) atomicAdd(cp.finished + MAX_CHAIN, 1);
+      if (cp.embed.table) {
+        // the first GEMM's per-token factors are sums over what ALL CTAs gathered
+        if (et == 0) {
+          bool there = false;
+          for (uint32_t spin = 0; spin < (1u << 22) && !there; ++spin) {
+            int seen;
+            asm volatile("ld.acquire.gpu.global.b32 %0, [%1];" : "=r"(seen) : "l"(cp.finished + MAX_CHAIN) : "memory");
+            there = seen - cp.fold_target >= 0;
+          }
+          wait_flag[0] = there && !*abort_flag;
+        }
+        epi_barrier();
+        ok = wait_flag[0] != 0;
+        epi_barrier();
+        __threadfence();
+      }
     }
     for (int ci = 0; ci < cp.n && ok; ++ci) {
     const GemmParams &p = cp.g[ci];
@@ -1058,7 +1112,7 @@ static void flush_chain(ouro_ctx *c) {
   for (int i = 0; i < cp.n; ++i) grid = std::max(grid, grid_for(s, cp.g[i].tiles, cp.g[i].kb));
   cp.finished = s.finished;
   for (int i = 0; i + 1 < cp.n; ++i) cp.target[i] = (s.finished_host[i] += cp.g[i].tiles);
-  if (cp.fold.part) cp.fold_target = (s.finished_host[MAX_CHAIN] += grid);
+  if (cp.fold.part || cp.embed.table) cp.fold_target = (s.finished_host[MAX_CHAIN] += grid);
   const bool per_kind = cp.n == 1 && c->prof_class >= OURO_PROF_QKV && c->prof_class <= OURO_PROF_HEAD;
   static const int kind_class[5] = {OURO_PROF_QKV, OURO_PROF_WO, OURO_PROF_GATEUP, OURO_PROF_DOWN, OURO_PROF_HEAD};
   {
@@ -1067,6 +1121,7 @@ static void flush_chain(ouro_ctx *c) {
   }
   cp.n = 0;
   cp.fold.part = nullptr;
+  cp.embed.table = nullptr;
 }
 
 // Adds a GEMM to the chain under construction; `last` launches the chain (something other than a GEMM follows).
@@ -1097,6 +1152,7 @@ void ouro_fast_reset(ouro_ctx *c, bool force) {
   FastState &s = c->fast->s;
   s.chain.n = 0;
   s.chain.fold.part = nullptr;
+  s.chain.embed.table = nullptr;
   if (!force && !s.dirty) return;
   cudaMemsetAsync(s.counters, 0, 2 * MAX_TILES * sizeof(int) + SPARE_BYTES, c->stream);
   for (int &v : s.finished_host) v = 0;
@@ -1104,35 +1160,6 @@ void ouro_fast_reset(ouro_ctx *c, bool force) {
 }
 void ouro_fast_mark_dirty(ouro_ctx *c) {
   if (c->fast) c->fast->s.dirty = true;
-}
-
-// Embedding rows into the residual stream, plus what the first norm's consumer needs: bf16(gain * x) and each
-// row's sum of squares (kept in tile 0 of the per-tile array, the other tiles zero).
-__global__ void embed_norm_kernel(const __nv_bfloat16 *E, const int32_t *tok, int d, const __nv_bfloat16 *gain, float *x,
-                                  __nv_bfloat16 *xb, float *ss, int ss_tiles, const int *rows_dev) {
-  pdl_trigger();
-  pdl_wait();
-  const int r = blockIdx.x;
-  if (rows_dev && r >= *rows_dev) return;          // the launch was sized for the largest possible block
-  const __nv_bfloat16 *src = E + (size_t)tok[r] * d;
-  float sq = 0.f;
-  for (int i = threadIdx.x; i < d; i += blockDim.x) {
-    float v = __bfloat162float(src[i]);
-    x[(size_t)r * d + i] = v;
-    xb[(size_t)r * d + i] = __float2bfloat16_rn(__bfloat162float(gain[i]) * v);
-    sq += v * v;
-  }
-  __shared__ float part[8];
-#pragma unroll
-  for (int o = 16; o; o >>= 1) sq += __shfl_xor_sync(0xffffffffu, sq, o);
-  if ((threadIdx.x & 31) == 0) part[threadIdx.x >> 5] = sq;
-  __syncthreads();
-  if (threadIdx.x == 0) {
-    float tot = 0.f;
-    for (int w = 0; w < (int)(blockDim.x >> 5); ++w) tot += part[w];
-    ss[r] = tot;
-  }
-  for (int i = 1 + threadIdx.x; i < ss_tiles; i += blockDim.x) ss[(size_t)i * OURO_MAX_ROWS + r] = 0.f;
 }
 
 // The row count of a candidate block may stay on the device when every kernel of the forward reads it from there:
@@ -1143,17 +1170,23 @@ bool ouro_fast_available(ouro_ctx *c, int which) {
   return d.head_dim == 64 || d.head_dim == 128;
 }
 
+// The embedding gather runs in front of the first layer's q,k,v GEMM, inside its launch.
 int ouro_fast_embed(ouro_ctx *c, int which, int rows) {
   if (!c->fast || !c->fast->s.m[which].ok) return OURO_ESTATE;
   ModelRt &M = c->m[which];
-  const ouro_model_desc &d = M.d;
-  c->fast->s.chain.n = 0;
-  c->fast->s.chain.fold.part = nullptr;
-  ProfScope ps(c, OURO_PROF_EMBED);
-  OURO_COUNT_LAUNCH();
-  launch_pdl(embed_norm_kernel, rows, 256, 0, c->stream, (const __nv_bfloat16 *)M.embed, (const int32_t *)M.blk.tok, (int)d.d_model,
-             (const __nv_bfloat16 *)M.attn_norm[0], c->a.x, (__nv_bfloat16 *)c->a.xn, c->fast->s.ss, (int)((d.d_model + TILE_N - 1) / TILE_N),
-             (const int *)(M.blk_rows_dev ? &c->st->n_rows : nullptr));
+  ChainParams &cp = c->fast->s.chain;
+  cp.n = 0;
+  cp.fold.part = nullptr;
+  ChainParams::Embed &e = cp.embed;
+  e.table = (const __nv_bfloat16 *)M.embed;
+  e.tok = M.blk.tok;
+  e.gain = (const __nv_bfloat16 *)M.attn_norm[0];
+  e.x = c->a.x;
+  e.xb = (__nv_bfloat16 *)c->a.xn;
+  e.ss = c->fast->s.ss;
+  e.rows_dev = c->cur_rows_dev;
+  e.rows = rows;
+  e.d = M.d.d_model;
   return OURO_OK;
 }
 
