@@ -120,7 +120,7 @@ def test_assemble_matches_oracle(gamma, beta, K, n_fill):
 
 # ------------------------------------------------------------------------------ forward logits
 
-def _verify_case(eng, W, desc, P, seed, L_prompt, tol_fn):
+def _verify_case(eng, W, desc, P, seed, L_prompt, tol_fn, full_block=False):
     rng = np.random.default_rng(seed)
     prompt = synth.prompt(seed, desc.vocab, L_prompt, 0.4, 4, 8)
     eng.reset()
@@ -129,11 +129,17 @@ def _verify_case(eng, W, desc, P, seed, L_prompt, tol_fn):
     ref_pool.apply(ob.prompt_ops(prompt, P.beta, P))
     d = rng.integers(0, desc.vocab, P.gamma).tolist()
     d[-1] = int(prompt[5])                     # a key that the seeded pool knows
+    if full_block:                             # K phrases with that key, so that the block has all its rows
+        grams = rng.integers(0, desc.vocab, (P.K, P.beta)).astype(np.int32)
+        grams[:, 0] = d[-1]
+        eng.phrase_update(grams)
+        for g in grams:
+            ref_pool.insert(g)
     eng.assemble_candidates(draft=d)
     tok, pos, grp, mask = eng.block_get()
     cands = ref_pool.lookup(d[-1], P.K)
     t2, p2, g2, vis = ob.build_block(len(prompt) - 1, prompt[-1], d, cands)
-    assert tok.tolist() == t2 and len(cands) >= 1
+    assert tok.tolist() == t2 and len(cands) >= 1 and (not full_block or len(t2) == P.block_max)
     am, logits = eng.verify_forward(want_logits=True)
     cache = tf.KVCache(desc)
     ob.prefill(W, cache, list(prompt[:-1]))
@@ -320,7 +326,11 @@ def c1():
     eng.close()
 
 
-@pytest.mark.parametrize("seed", [0, 1, 2])
+C1_SEEDS = [0, 1, 2, 4]
+_c1_seen = {}
+
+
+@pytest.mark.parametrize("seed", C1_SEEDS)
 def test_generate_c1_matches_oracle_and_vanilla(c1, seed):
     eng, W, Wd = c1
     prompt = synth.prompt(seed, C1T.vocab, C1R["n"], C1R["copy_frac"], *C1R["span"])
@@ -339,6 +349,14 @@ def test_generate_c1_matches_oracle_and_vanilla(c1, seed):
     assert stats["candidates"] == sum(rstats["n_cand"])
     assert pool_gpu[0] == [list(p) for _, p in trace[-1]["pool"]]    # same pool, same order
     assert pool_gpu[1] == [s for s, _ in trace[-1]["pool"]]
+    _c1_seen[seed] = (sum(rstats["A"]), stats["suffix_tokens"], stats["target_calls"])
+    if len(_c1_seen) == len(C1_SEEDS):
+        # The early-exit draft (one of the target's two layers) agrees with the target only now and then: seed 0 runs
+        # with block efficiency 1 (no draft token is ever accepted).  Over the seeds draft tokens must have been
+        # accepted, or this comparison would not exercise acceptance at all.  Phrase suffixes are never accepted
+        # with these natural drafts; the replayed-draft test below asserts suffix_tokens > 0.
+        assert sum(v[0] for v in _c1_seen.values()) > 20, _c1_seen
+        assert any(v[2] < gen for v in _c1_seen.values()), _c1_seen
 
 
 def test_teacher_forced_steps_c1(c1):
@@ -679,3 +697,123 @@ def test_verify_logits_bf16_gqa_head_dim_128(seed, L_prompt):
 def test_verify_logits_bf16_widest_blocks(gamma, beta, K, L_prompt):
     """The widest block (128 rows: four rounds of query rows) and the most groups (16 candidates + trunk)."""
     _gqa_case(synth.DecodeParams(gamma, beta, K, 2, 32, seed_prompt=False), 5, L_prompt)
+
+
+# ------------------------------------------------------------------ full-width shapes against the oracle
+
+def _oracle_weights(desc, w):
+    return tf.Weights(desc, {n: (t.cpu() if n != "layers" else [{a: b.cpu() for a, b in lw.items()} for lw in t]) for n, t in w.items()})
+
+
+@pytest.mark.parametrize("name,K", [("C4", 8), ("C5", 4)])
+def test_verify_logits_full_width_one_layer(name, K):
+    """One decoder layer + LM head at the widths of the 34B- and 70B-shaped targets (d 7168 / 8192, 56 / 64 query
+    heads on 8 kv heads, FFN 20480 / 28672, vocabulary 64000 / 32000): the candidate block (69 / 37 rows) on a
+    prefilled cache, logits, greedy tokens and appended K/V against the oracle."""
+    T, _, P, _ = synth.config(name)
+    desc = dataclasses.replace(T, n_layers=1, max_seq=448)
+    assert P.K == K and P.block_max == 1 + 4 + K * 8
+    w = synth.model_weights(desc, 0, device="cuda:0")
+    eng = binding.Engine(desc, w, P)
+    W = _oracle_weights(desc, w)
+    _verify_case(eng, W, desc, P, 2, 150, _bf16_tol, full_block=True)
+    eng.close()
+
+
+def test_teacher_forced_bf16_four_layer_7b_stack():
+    """Four 7B-shaped layers (d 4096, FFN 11008, vocabulary 32000), bf16, ten decoding steps with replayed drafts and
+    phrases: at every step the oracle evaluates the same block on the same history - logits within the bf16 bound,
+    greedy tokens equal wherever the oracle's margin allows, acceptance / compaction / pool bit exact."""
+    T, _, P, R = synth.config("C3")
+    desc = dataclasses.replace(T, n_layers=4, max_seq=320)
+    w = synth.model_weights(desc, 0, device="cuda:0")
+    eng = binding.Engine(desc, w, P)
+    W = _oracle_weights(desc, w)
+    prompt = synth.prompt(1, desc.vocab, 48, R["copy_frac"], 4, 8)
+    van, _ = eng.generate_vanilla(prompt, 96)
+    truth = np.concatenate([prompt, van, np.zeros(64, dtype=np.int32)])
+    eng.reset(); eng.prefill(prompt)
+    cache = tf.KVCache(desc); ob.prefill(W, cache, list(prompt[:-1]))
+    pool = oracle_pool(P); pool.apply(ob.prompt_ops(prompt, P.beta, P))
+    seq = prompt.tolist()
+    worst, suffix_tokens, full = 0.0, 0, 0
+    for step in range(10):
+        L = cache.length
+        d = synth.corrupt_drafts(5, truth, len(seq), P.gamma, desc.vocab, 0.10, 0.03, step).tolist()
+        grams = np.empty((P.K, P.beta), dtype=np.int32)
+        for j in range(P.K):                                   # phrases that continue the draft, more or less corrupted
+            grams[j, 0] = d[-1]
+            grams[j, 1:] = synth.corrupt_drafts(11 + j, truth, len(seq) + P.gamma, P.S, desc.vocab, 0.08 * (j + 1), 0.0, step)
+        eng.phrase_update(grams[::-1])
+        for g in grams[::-1]:
+            pool.insert(g)
+        eng.assemble_candidates(draft=d)
+        tok = eng.block_get()[0].tolist()
+        cands = pool.lookup(d[-1], P.K)
+        tokens, pos, group, vis = ob.build_block(L, seq[-1], d, cands)
+        assert tok == tokens
+        am, logits = eng.verify_forward(want_logits=True)
+        want = tf.forward(W, cache, tokens, pos, vis)
+        got = logits[: len(tokens)].cpu().numpy().astype(np.float64)
+        rel = np.abs(got - want).max(axis=1) / np.abs(want).max(axis=1)
+        worst = max(worst, rel.max())
+        assert rel.max() < BF16_REL, (step, rel.max())
+        err = np.abs(got - want).max(axis=1)
+        srt = np.sort(want, axis=1)
+        safe = (srt[:, -1] - srt[:, -2]) > 2 * err + 1e-12
+        o = am[: len(tokens)].cpu().numpy()
+        assert np.array_equal(o[safe], tf.argmax_rows(want)[safe])
+        n, chosen, A, acc = eng.accept_and_compact()
+        A2, j2, m2, acc2 = ob.accept(tokens, o.tolist(), P.gamma, P.S, len(cands))
+        assert (n, chosen, A, acc.tolist()) == (len(acc2), j2, A2, acc2)
+        ob.compact(cache, L, P.gamma, P.S, A2, j2, m2)
+        seq += acc2
+        pool.apply(ob.harvest_ops(tokens, o.tolist(), P.gamma, P.S, len(cands), A2, seq, len(acc2), P))
+        assert gpu_pool_rows(eng) == pool_rows(pool)
+        Ln = cache.length
+        kv_tol = 2e-2 * max(np.abs(cache.k[:, :Ln]).max(), np.abs(cache.v[:, :Ln]).max())
+        assert np.abs(eng.tm.k_cache[:, :Ln].float().cpu().numpy() - cache.k[:, :Ln]).max() < kv_tol
+        assert np.abs(eng.tm.v_cache[:, :Ln].float().cpu().numpy() - cache.v[:, :Ln]).max() < kv_tol
+        suffix_tokens += m2 if j2 >= 0 else 0
+        full += A2 == P.gamma
+        assert seq[len(prompt):] == van[: len(seq) - len(prompt)].tolist()      # the accepted text is the greedy text
+    assert full >= 3 and suffix_tokens > 0, (full, suffix_tokens)
+    eng.close()
+
+
+@pytest.mark.parametrize("rows", [1, 37])
+def test_exact_logit_ties_take_the_smallest_id(rows):
+    """Identical rows of the LM head give bit-identical logits when they are accumulated the same way: inside one
+    128-entry tile of the head GEMM, or in different tiles that one CTA handles over the whole K range (a tile whose
+    K range is split across CTAs adds its partial sums in another order, so it rounds differently).  The greedy
+    choice among such equals must be the smallest id - for a single row (plain decoding) and for a candidate block."""
+    desc = synth.ModelDesc(1, 256, 4, 4, 64, 512, 32000, 192, "bf16")       # 250 head tiles: whole and split ones
+    w = synth.model_weights(desc, 4, device="cuda:0")
+    P = synth.DecodeParams(4, 9, 4, 16, 8, seed_prompt=False)
+    eng = binding.Engine(desc, w, P)
+    tokens = (np.arange(rows) * 7 + 3).astype(np.int32)
+    eng.assemble_causal(binding.OURO_TARGET, tokens)
+    _, lg = eng.verify_forward(want_logits=True)
+    base = lg[:rows].clone()
+    # a head row that wins for every token: a large multiple of the mean normalised activation direction is not
+    # available from outside, so take the current winner's row of token 0 and scale it up
+    win_id = int(base[0].argmax())
+    boosted = (w["lm_head"][win_id].float() * 4.0).to(torch.bfloat16)
+    # 250 tiles on 148 CTAs: tiles 0..147 are handled whole, 148..249 are split along K
+    for ids in ((700, 731, 5000), (18900, 130, 131), (19050, 19000)):
+        saved = {i: w["lm_head"][i].clone() for i in ids}
+        for i in ids:
+            w["lm_head"][i] = boosted
+        am, lg = eng.verify_forward(want_logits=True)
+        torch.cuda.synchronize()
+        vals = {float(lg[0, i]) for i in ids}
+        assert len(vals) == 1 and int(lg[0].argmax()) in ids, (vals, int(lg[0].argmax()))
+        assert int(am[0]) == min(ids)
+        for r in range(rows):                              # every row: the choice is the smallest index among the maxima
+            mx = lg[r].max()
+            assert int(am[r]) == int(torch.nonzero(lg[r] == mx)[0])
+        am2, _ = eng.verify_forward()                      # and the same without materialised logits
+        assert torch.equal(am2[:rows], am[:rows])
+        for i in ids:
+            w["lm_head"][i] = saved[i]
+    eng.close()
