@@ -217,6 +217,13 @@ enum {
 /* Number of kernels this library has launched in this process (all contexts), for launch accounting. */
 uint64_t ouro_kernel_launches(void);
 int ouro_profile_enable(ouro_ctx *ctx, int kernel_class);
+/* Test aid for the give-up path of the bounded device-side waits (no counterpart in the paper).  A GEMM tile whose K
+ * range is split across CTAs is finished once all contributors have published their partial sums; the waiting thread
+ * polls a counter at most `polls` times (default 1 << 22; negative restores the default).  0 makes the wait give up
+ * at once: the kernels return normally, the status word is raised, the next call that reads results back
+ * (ouro_accept_and_compact, ouro_generate, ouro_generate_vanilla) returns OURO_ETIMEOUT, and ouro_reset makes the
+ * context usable again.  OURO_ESTATE when the context does not run the tensor-core kernels. */
+int ouro_debug_set_wait_limit(ouro_ctx *ctx, int64_t polls);
 int ouro_profile_read(ouro_ctx *ctx, float *ms_total, int32_t *launches);
 
 /* (The paper has no counterpart to this call; it exists for deployment reasons only.)

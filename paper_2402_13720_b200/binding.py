@@ -79,6 +79,7 @@ _SIGNATURES = {
     "ouro_kernel_launches": (C.c_uint64, []),
     "ouro_lm_head_static": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p]),
     "ouro_profile_enable": (C.c_int, [C.c_void_p, C.c_int]),
+    "ouro_debug_set_wait_limit": (C.c_int, [C.c_void_p, C.c_int64]),
     "ouro_profile_read": (C.c_int, [C.c_void_p, _F32P, _I32P]),
     "ouro_generate": (C.c_int, [C.c_void_p, _I32P, C.c_int32, C.c_int32, C.c_int32, _I32P, _I32P, C.POINTER(StatsC)]),
     "ouro_generate_vanilla": (C.c_int, [C.c_void_p, _I32P, C.c_int32, C.c_int32, _I32P, _I32P, C.POINTER(StatsC)]),
@@ -331,6 +332,9 @@ class Engine:
         ms, n = C.c_float(), C.c_int32()
         self._ck(self.L.ouro_profile_read(self.ctx, C.byref(ms), C.byref(n)))
         return ms.value, n.value
+
+    def set_wait_limit(self, polls):
+        self._ck(self.L.ouro_debug_set_wait_limit(self.ctx, int(polls)))
 
     # ---- loops -------------------------------------------------------------------------------
     def generate(self, prompt, max_new, keep_pool=False):

@@ -824,7 +824,12 @@ extern "C" int ouro_generate_vanilla(ouro_ctx *c, const int32_t *prompt, int32_t
   }
   CK(cudaEventRecord(c->ev[5], s));
   CK(cudaMemcpyAsync(out, c->seq_dev + base, (size_t)n * 4, cudaMemcpyDeviceToHost, s));
+  CK(cudaMemcpyAsync(c->pin, &c->st->status, sizeof(int32_t), cudaMemcpyDeviceToHost, s));
   CK(cudaStreamSynchronize(s));
+  if (c->pin[0] != 0) {
+    ouro_fast_mark_dirty(c);
+    return fail(c, OURO_ETIMEOUT, "device status word " + std::to_string(c->pin[0]));
+  }
   CK(cudaEventElapsedTime(&st.ms_total, c->ev[0], c->ev[5]));
   st.ms_target = st.ms_total;
   c->seq.insert(c->seq.end(), out, out + n);

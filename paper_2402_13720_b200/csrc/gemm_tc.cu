@@ -100,6 +100,7 @@ struct GemmParams {
   int *done;          // [tiles] contributors that finished their share, zero between launches
   int *status;        // context status word
   int trace_id;           // which GEMM of the layer this is (timeline builds only)
+  uint32_t wait_limit;    // polls of a partial-tile wait before it gives up (1 << 22 unless a test shortens it)
 };
 
 // A chain of GEMMs run by one persistent launch, each consuming what the one before produced (output projection ->
@@ -142,10 +143,11 @@ __device__ __forceinline__ void mbar_expect_tx(uint64_t *bar, uint32_t bytes) {
 __device__ __forceinline__ void mbar_arrive(uint64_t *bar) {
   asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
-// Bounded wait: false when the limit ran out (the caller raises the status word and drains).
-__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity) {
+// Bounded wait: false when the limit ran out or another warp of the CTA has given up (the caller raises the status
+// word and drains).
+__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volatile int *abort_flag, uint32_t limit = SPIN_LIMIT) {
   uint32_t addr = smem_u32(bar);
-  for (uint32_t i = 0; i < SPIN_LIMIT; ++i) {
+  for (uint32_t i = 0; i < limit; ++i) {
     uint32_t ok;
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
@@ -155,6 +157,7 @@ __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity) {
         : "r"(addr), "r"(parity)
         : "memory");
     if (ok) return true;
+    if ((i & 255) == 255 && abort_flag && *abort_flag) return false;
   }
   return false;
 }
@@ -233,13 +236,17 @@ __device__ __forceinline__ void locate(const GemmParams &p, int tile, int &seg, 
 }
 
 // Bounded wait until GEMM `i` of the chain has finished all its tiles (acquire).
-__device__ __forceinline__ bool chain_wait(const ChainParams &cp, int i) {
-  for (uint32_t spin = 0; spin < (1u << 22); ++spin) {
+__device__ __forceinline__ bool counter_wait(const int *counter, int target, const int *status, uint32_t limit) {
+  for (uint32_t spin = 0; spin < limit; ++spin) {
     int seen;
-    asm volatile("ld.acquire.gpu.global.b32 %0, [%1];" : "=r"(seen) : "l"(cp.finished + i) : "memory");
-    if (seen - cp.target[i] >= 0) return true;
+    asm volatile("ld.acquire.gpu.global.b32 %0, [%1];" : "=r"(seen) : "l"(counter) : "memory");
+    if (seen - target >= 0) return true;
+    if ((spin & 15) == 15 && *(volatile const int *)status != 0) return false;   // some CTA has given up: nobody waits on
   }
   return false;
+}
+__device__ __forceinline__ bool chain_wait(const ChainParams &cp, int i) {
+  return counter_wait(cp.finished + i, cp.target[i], cp.g[0].status, 1u << 22);
 }
 
 __global__ void __launch_bounds__(THREADS, 1) gemm_tc_kernel(const __grid_constant__ ChainParams cp) {
@@ -256,6 +263,7 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_tc_kernel(const __grid_consta
   uint32_t *tmem_base_p = (uint32_t *)(bars + 36);
   volatile int *abort_flag = (volatile int *)(bars + 37);
   volatile int *wait_flag = (volatile int *)(bars + 39);   // [0..1]: outcome of an accumulator wait; [2]: a fix-up gave up; [4..5]: outcome of a fix-up group's wait
+  uint64_t *drain_bar = bars + 44;                          // give-up path: "every contraction issued so far has completed"
   float *rs = (float *)(bars + 48);                         // [128] per-token factor 1/rms of the consumed activations
   int *spos = (int *)(rs + OURO_MAX_ROWS);                  // [128] token positions (rotary table rows), QKV epilogue
 
@@ -273,6 +281,7 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_tc_kernel(const __grid_consta
       mbar_init(&acc_full[a], 1);
       mbar_init(&acc_empty[a], 4);
     }
+    mbar_init(drain_bar, 1);
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -285,6 +294,7 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_tc_kernel(const __grid_consta
   __syncthreads();
   fence_after_sync();
   const uint32_t tmem_base = *tmem_base_p;
+  uint32_t n_issued = 0;                           // producer lanes: stages they have issued copies into
 
   if (warp == 0) {
     // ---------------------------------------------------------------- TMA producer
@@ -312,7 +322,7 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_tc_kernel(const __grid_consta
       while (ok && w.next(s)) {
         for (int kb = s.kb0; kb < s.kb1 && ok; ++kb, ++n) {
           int st = n % n_stages;
-          if (n >= (uint32_t)n_stages) ok = mbar_wait(&empty[st], ((n / n_stages) - 1) & 1) && !*abort_flag;
+          if (n >= (uint32_t)n_stages) ok = mbar_wait(&empty[st], ((n / n_stages) - 1) & 1, abort_flag) && !*abort_flag;
           if (!ok) break;
           issue(s, kb, st);
         }
@@ -320,6 +330,7 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_tc_kernel(const __grid_consta
       TRACE(8);
       }
       if (!ok) { *abort_flag = 1; atomicExch(p0.status, 1); }
+      n_issued = n;
     }
   } else if (warp == 6) {
     // ---------------------------------------------------------------- activation producer
@@ -328,12 +339,7 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_tc_kernel(const __grid_consta
       uint32_t n = 0;
       bool ok = true;
       if (cp.fold.part || cp.embed.table) {        // ... once every CTA has done its share of the fold / the gather
-        ok = false;
-        for (uint32_t spin = 0; spin < (1u << 22) && !ok; ++spin) {
-          int seen;
-          asm volatile("ld.acquire.gpu.global.b32 %0, [%1];" : "=r"(seen) : "l"(cp.finished + MAX_CHAIN) : "memory");
-          ok = seen - cp.fold_target >= 0;
-        }
+        ok = counter_wait(cp.finished + MAX_CHAIN, cp.fold_target, p0.status, 1u << 22);
         asm volatile("fence.proxy.async;" ::: "memory");
       }
       for (int ci = 0; ci < cp.n && ok; ++ci) {
@@ -351,7 +357,7 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_tc_kernel(const __grid_consta
         while (ok && w.next(s)) {
           for (int kb = s.kb0; kb < s.kb1 && ok; ++kb, ++n) {
             int st = n % n_stages;
-            if (n >= (uint32_t)n_stages) ok = mbar_wait(&empty[st], ((n / n_stages) - 1) & 1) && !*abort_flag;
+            if (n >= (uint32_t)n_stages) ok = mbar_wait(&empty[st], ((n / n_stages) - 1) & 1, abort_flag) && !*abort_flag;
             if (!ok) break;
             mbar_expect_tx(&full[st], b_bytes);
             tma_load_2d(ring + (size_t)st * stage_bytes + A_BYTES, &p.b, &full[st], kb * BLOCK_K, 0, HINT_EVICT_LAST);
@@ -359,6 +365,7 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_tc_kernel(const __grid_consta
         }
       }
       if (!ok) { *abort_flag = 1; atomicExch(p0.status, 1); }
+      n_issued = n;
     }
   } else if (warp == 1) {
     // ---------------------------------------------------------------- MMA issuer
@@ -373,13 +380,13 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_tc_kernel(const __grid_consta
       bool first = true;
       while (ok && w.next(s)) {
         int a = item & 1;
-        if (item >= 2) ok = mbar_wait(&acc_empty[a], ((item >> 1) - 1) & 1) && !*abort_flag;
+        if (item >= 2) ok = mbar_wait(&acc_empty[a], ((item >> 1) - 1) & 1, abort_flag) && !*abort_flag;
         if (!ok) break;
         fence_after_sync();
         uint32_t tmem_d = tmem_base + a * acc_cols;
         for (int kb = s.kb0; kb < s.kb1; ++kb, ++n) {
           int st = n % n_stages;
-          ok = mbar_wait(&full[st], (n / n_stages) & 1) && !*abort_flag;
+          ok = mbar_wait(&full[st], (n / n_stages) & 1, abort_flag) && !*abort_flag;
           if (!ok) break;
           if (first) { TRACE(2); first = false; }
           fence_after_sync();
@@ -440,15 +447,7 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_tc_kernel(const __grid_consta
       if (et == 0) atomicAdd(cp.finished + MAX_CHAIN, 1);
       if (cp.embed.table) {
         // the first GEMM's per-token factors are sums over what ALL CTAs gathered
-        if (et == 0) {
-          bool there = false;
-          for (uint32_t spin = 0; spin < (1u << 22) && !there; ++spin) {
-            int seen;
-            asm volatile("ld.acquire.gpu.global.b32 %0, [%1];" : "=r"(seen) : "l"(cp.finished + MAX_CHAIN) : "memory");
-            there = seen - cp.fold_target >= 0;
-          }
-          wait_flag[0] = there && !*abort_flag;
-        }
+        if (et == 0) wait_flag[0] = counter_wait(cp.finished + MAX_CHAIN, cp.fold_target, p0.status, 1u << 22) && !*abort_flag;
         epi_barrier();
         ok = wait_flag[0] != 0;
         epi_barrier();
@@ -476,12 +475,7 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_tc_kernel(const __grid_consta
     // Returns false when the wait gave up.
     auto others_there = [&](int tile, int n, int gi, int grp, int G) -> bool {
       if (gi == 0) {
-        int seen = 0;
-        for (uint32_t i = 0; i < (1u << 22); ++i) {
-          asm volatile("ld.acquire.gpu.global.b32 %0, [%1];" : "=r"(seen) : "l"(p.counters + tile) : "memory");
-          if (seen >= n) break;
-        }
-        wait_flag[4 + grp] = seen >= n && !*abort_flag;
+        wait_flag[4 + grp] = counter_wait(p.counters + tile, n, p.status, p.wait_limit) && !*abort_flag;
         TRACE(6);
       }
       if (G == 128) epi_barrier(); else group_barrier(grp);
@@ -790,7 +784,7 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_tc_kernel(const __grid_consta
       if (s.n_contrib == 1 && n_pend > 0) run_fixups();
       if (!ok) break;
       // one thread waits (bounded) and tells the others, so that all 128 leave the loop together
-      if (et == 0) wait_flag[a] = mbar_wait(&acc_full[a], (item >> 1) & 1) && !*abort_flag;
+      if (et == 0) wait_flag[a] = mbar_wait(&acc_full[a], (item >> 1) & 1, abort_flag) && !*abort_flag;
       epi_barrier();
       ok = wait_flag[a] != 0;
       if (!ok) break;
@@ -885,6 +879,21 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_tc_kernel(const __grid_consta
   // ------------------------------------------------------------------ teardown
   fence_before_sync();
   __syncthreads();
+  if (*abort_flag && lane == 0 && (warp == 0 || warp == 6)) {
+    // Somebody gave up: copies this lane issued may still be landing in this CTA's shared memory.  Wait (bounded) for
+    // the last one of every stage before the CTA leaves; a stage whose other half was never requested cannot
+    // complete its phase, which the limit covers (the bytes themselves arrive within microseconds).
+    for (int st = 0; st < n_stages; ++st) {
+      if (n_issued <= (uint32_t)st) continue;
+      const uint32_t last = ((n_issued - 1 - st) / n_stages) * n_stages + st;      // last copy issued into this stage
+      mbar_wait(&full[st], (last / n_stages) & 1, nullptr, 1u << 14);
+    }
+  }
+  if (*abort_flag && warp == 1 && lane == 0) {     // ... and no contraction may still be running when TMEM is given back
+    mma_commit(drain_bar);
+    mbar_wait(drain_bar, 0, nullptr, 1u << 16);
+  }
+  __syncthreads();
   if (warp == 1) {
     fence_after_sync();
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)(2 * acc_cols)));
@@ -934,6 +943,7 @@ struct FastState {
   int chain_kind[MAX_CHAIN] = {0, 0, 0, 0};
   bool fuse = true;             // run consecutive GEMMs as one launch
   bool dirty = false;           // a bounded wait gave up: counters must be cleared before the next launch
+  uint32_t wait_limit = 1u << 22;   // polls of a partial-tile wait (ouro_debug_set_wait_limit)
 };
 constexpr int MAX_TILES = 4096;
 constexpr int SPARE_BYTES = 2048;          // behind the tile counters: chain counters [0, 64), attention arrival counters [64, 512)
@@ -1138,6 +1148,7 @@ static void push_gemm(ouro_ctx *c, GemmParams &p, int kind, const CUtensorMap *x
   p.status = &c->st->status;
   p.rows_dev = c->cur_rows_dev;
   p.trace_id = kind;
+  p.wait_limit = s.wait_limit;
   if (s.chain.n > 0 && s.chain.g[0].rows != rows) flush_chain(c);   // cannot happen inside one forward
   s.chain_kind[s.chain.n] = kind;
   s.chain.g[s.chain.n++] = p;
@@ -1160,6 +1171,12 @@ void ouro_fast_reset(ouro_ctx *c, bool force) {
 }
 void ouro_fast_mark_dirty(ouro_ctx *c) {
   if (c->fast) c->fast->s.dirty = true;
+}
+extern "C" int ouro_debug_set_wait_limit(ouro_ctx *c, int64_t polls) {
+  if (!c) return OURO_EINVAL;
+  if (!c->fast) return OURO_ESTATE;
+  c->fast->s.wait_limit = polls < 0 ? (1u << 22) : (uint32_t)std::min<int64_t>(polls, 1u << 22);
+  return OURO_OK;
 }
 
 // The row count of a candidate block may stay on the device when every kernel of the forward reads it from there:
@@ -1455,6 +1472,7 @@ extern "C" int ouro_lm_head_static(const void *x_dev, const void *lm_head_dev, i
   p.ldo = vocab;
   p.tile_max = (float *)(base + NA_OFF_TMAX);
   p.tile_arg = (int *)(base + NA_OFF_TARG);
+  p.wait_limit = 1u << 22;
   p.scratch = (float *)base;
   p.counters = (int *)(base + NA_OFF_COUNTERS);
   p.done = p.counters + NA_MAX_TILES;

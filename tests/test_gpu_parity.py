@@ -817,3 +817,36 @@ def test_exact_logit_ties_take_the_smallest_id(rows):
         for i in ids:
             w["lm_head"][i] = saved[i]
     eng.close()
+
+
+# ------------------------------------------------------------------ a bounded device-side wait that runs out
+
+def test_bounded_wait_gives_up_and_the_context_recovers():
+    """The wait of a split-K tile for its other contributors is bounded.  With the bound set to zero polls it runs out
+    at once (nothing is made to fault: the kernels return normally with the status word raised): the call that reads
+    results back reports OURO_ETIMEOUT, plain decoding reports it too, and after a reset the same context computes
+    oracle-equal logits again."""
+    P = synth.DecodeParams(4, 9, 4, 16, 8)
+    eng, W = make(MIDB, P, 2)                      # d 256: every q,k,v tile is split four ways
+    _verify_case(eng, W, MIDB, P, 2, 40, _bf16_tol)
+    eng.accept_and_compact()
+    prompt = synth.prompt(2, MIDB.vocab, 40, 0.4, 4, 8)
+    eng.set_wait_limit(0)
+    eng.reset(); eng.prefill(prompt[:2])           # one causal row: raises the status word on the device
+    eng.assemble_candidates(draft=[1, 2, 3, int(prompt[5])])
+    eng.verify_forward()
+    with pytest.raises(binding.OuroError) as e:
+        eng.accept_and_compact()
+    assert e.value.status == binding.OURO_ETIMEOUT
+    with pytest.raises(binding.OuroError) as e:
+        eng.generate_vanilla(prompt, 4)
+    assert e.value.status == binding.OURO_ETIMEOUT
+    eng.set_wait_limit(-1)
+    _verify_case(eng, W, MIDB, P, 2, 40, _bf16_tol)     # reset + prefill + verify: as before the give-up
+    eng.accept_and_compact()
+    van, _ = eng.generate_vanilla(prompt, 12)
+    eng.set_drafter(lambda seq, g, step: [int(van[min(len(seq) - len(prompt) + i, 11)]) for i in range(g)])
+    out, _ = eng.generate(prompt, 12)
+    eng.set_drafter(None)
+    assert len(van) == 12 and np.array_equal(out, van)
+    eng.close()
