@@ -24,8 +24,7 @@ import numpy as np
 import torch
 
 ROOT = os.path.dirname(os.path.abspath(__file__))
-GEMM_TRAFFIC_BYTES = 138.3e6          # dram read + write per gemm_tc_kernel launch, mean of the step's five launches (ncu)
-GEMM_TRAFFIC_REV = "996ec95f789f5ff6"  # kernel_rev() of the source the counters were taken on
+GEMM_PROFILE = os.path.join(ROOT, "profiles", "gemm_tc_kernel_verify_step_c2.md")
 
 
 def kernel_rev():
@@ -36,12 +35,24 @@ def kernel_rev():
     cut = src.find(b"host side")
     return hashlib.sha256(src[:cut] if cut > 0 else src).hexdigest()[:16]
 
+
+def profiled_traffic():
+    """DRAM bytes (read + write) per gemm_tc_kernel launch from the ncu capture summarised in profiles/: the summary
+    carries a line `traffic_bytes_per_launch: <number> kernel_rev: <hash>`; the figure counts only while the kernel's
+    device code still has that hash."""
+    import re
+    try:
+        m = re.search(r"traffic_bytes_per_launch:\s*([0-9.e+]+)\s+kernel_rev:\s*([0-9a-f]+)", open(GEMM_PROFILE).read())
+    except OSError:
+        return None
+    return float(m.group(1)) if m and m.group(2) == kernel_rev() else None
+
 from paper_2402_13720_b200 import synth  # noqa: E402
 
 METRIC, UNIT = "verify_step_hbm_throughput", "GB/s"
 SEED = 0
 PENDING = 17
-PROF_CLASSES = ("qkv", "attention", "wo", "gateup", "down", "head")
+PROF_CLASSES = ("qkv", "attention", "wo", "gateup", "down", "head")     # "gemm": every launch of the weight-streaming kernel
 
 
 # ------------------------------------------------------------------------------ workload
@@ -98,9 +109,8 @@ class GpuWorkload:
         e.set_state(self.L, PENDING)
         if host_inputs:                               # end-to-end: the step's inputs start in pinned host memory
             e.draft_tokens.copy_(self.draft_pinned, non_blocking=True)
-        e.assemble_candidates()
-        e.verify_forward()
-        return e.accept_and_compact()                 # returns host values: a device->host read per step
+        return e.verify_step()                        # lookup + packing, forward, acceptance + compaction + harvest;
+                                                      # returns host values: a device->host read per step
 
     def check(self):
         e = self.eng
@@ -368,6 +378,53 @@ def run_generate(args, device):
     eng.close()
 
 
+def generation_summary(device, tokens):
+    """BASELINE's other half: generated tokens/s at batch 1 on the 7B-shaped target with the 1.1B-shaped draft model
+    (configs[2]), plain greedy decoding against Ouroboros with replayed drafts (middle agreement level) without and
+    with the replayed phrase source.  A short run: `tokens` generated tokens per mode."""
+    import dataclasses
+    from paper_2402_13720_b200 import binding
+    T, D, P, R = synth.config("C3")
+    wt = synth.model_weights(T, SEED, device=device)
+    wd = synth.model_weights(D, SEED + 100, device=device)
+    eng = binding.Engine(T, wt, P, D, wd, device=device)
+    prompt = synth.prompt(SEED, T.vocab, R["n"], R["copy_frac"], *R["span"])
+    eng.generate_vanilla(prompt, 8)
+    van, vs = eng.generate_vanilla(prompt, tokens)
+    truth = np.concatenate([prompt, van, np.zeros(64, dtype=np.int32)])
+    out = {"config": f"configs[2]: 7B-shaped target, 1.1B-shaped draft, bf16, prompt {R['n']}, {tokens} tokens, gamma {P.gamma}, "
+                     f"beta {P.beta}, K {P.K}",
+           "vanilla": {"tokens_per_s": round(len(van) / (vs["ms_total"] * 1e-3), 1)}}
+
+    def run(name, drafter):
+        eng.set_drafter(drafter)
+        o, st = eng.generate(prompt, tokens)
+        eng.set_drafter(None)
+        out[name] = {"tokens_per_s": round(len(o) / (st["ms_total"] * 1e-3), 1),
+                     "vs_vanilla": round(len(o) / (st["ms_total"] * 1e-3) / out["vanilla"]["tokens_per_s"], 3),
+                     "tokens_per_target_call": round(len(o) / st["target_calls"], 2), "suffix_tokens": st["suffix_tokens"],
+                     "ms_target_per_call": round(st["ms_target"] / st["target_calls"], 3),
+                     "ms_draft_per_step": round(st["ms_draft"] / st["target_calls"], 3),
+                     "identical_to_vanilla": bool(np.array_equal(o, van))}
+
+    def drafts(seq, g, step):
+        return synth.corrupt_drafts(SEED + 7, truth, len(seq), g, T.vocab, 0.12, 0.03, step)
+
+    def drafts_and_phrases(seq, g, step):
+        d = drafts(seq, g, step)
+        grams = np.empty((P.K, P.beta), dtype=np.int32)
+        for j in range(P.K):
+            grams[j, 0] = d[-1]
+            grams[j, 1:] = synth.corrupt_drafts(SEED + 11 + j, truth, len(seq) + g, P.S, T.vocab, 0.08 * (j + 1), 0.0, step)
+        eng.phrase_update(grams[::-1])
+        return d
+
+    run("replayed_drafts", drafts)
+    run("replayed_drafts_and_phrases", drafts_and_phrases)
+    eng.close()
+    return out
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -376,6 +433,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--cache-len", type=int, default=4096)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-generation", action="store_true", help="skip the short whole-model generation summary")
+    ap.add_argument("--generation-tokens", type=int, default=96)
     ap.add_argument("--generate", default=None, choices=["C1", "C3", "C4", "C5"],
                     help="instead of the verify-step benchmark: whole generation on that configuration "
                          "(vanilla greedy vs Ouroboros, natural and replayed drafts), one JSON line")
@@ -422,10 +481,13 @@ def main():
     value = total_bytes / (ms * 1e-3) / 1e9
     e2e = total_bytes / (ms_e2e * 1e-3) / 1e9
 
-    # per-kernel-class device time of the forward, events on the library's own stream
+    # per-kernel-class device time of the forward, events on the library's own stream.  "gemm" brackets every launch
+    # of the weight-streaming kernel as the forward really runs it (two launches per step: q,k,v with the embedding
+    # gather; output projection + gate/up + down + LM head as one chain).  The per-GEMM classes are diagnostics: while
+    # one of them is timed, each GEMM is launched alone.
     prof = {}
     psteps = min(args.steps, 200)
-    for cls in PROF_CLASSES + ("forward",):
+    for cls in PROF_CLASSES + ("gemm", "forward"):
         wl.eng.profile_enable(cls)
         for _ in range(psteps):
             wl.step()
@@ -438,22 +500,22 @@ def main():
     except Exception:
         pass
     peak, peak_kind = (peaks["hbm_gbs"], "measured") if "hbm_gbs" in peaks else (6650.0, "fallback")
-    # The dominant kernel is the weight-streaming GEMM (one kernel, five launches per layer + head pass).
+    # The dominant kernel is the weight-streaming GEMM: its launches of one step stream every weight matrix once.
     gemm = ("qkv", "wo", "gateup", "down", "head")
-    gemm_ms = sum(prof[c][0] * prof[c][1] for c in gemm)
-    gemm_launches = sum(prof[c][1] for c in gemm)
-    gemm_bytes = sum(wl.bytes["per_class"][c] * prof[c][1] for c in gemm)
+    gemm_launches = prof["gemm"][1]
+    gemm_ms = prof["gemm"][0] * gemm_launches
+    gemm_bytes = sum(wl.bytes["per_class"][c] for c in gemm) * wl.m.n_layers - (wl.m.n_layers - 1) * wl.bytes["per_class"]["head"]
     achieved = gemm_bytes / (gemm_ms * 1e-3) / 1e9 if gemm_ms > 0 else 0.0
     fwd_ms = prof["forward"][0]
-    # DRAM bytes per launch (read + write) of the five GEMM launches from one ncu capture of this workload
-    # (profiles/gemm_tc_kernel_verify_step_c2.md); it belongs to GEMM_TRAFFIC_REV of the kernel source and
-    # is reported as null once the kernel has changed since.
-    traffic = GEMM_TRAFFIC_BYTES if kernel_rev() == GEMM_TRAFFIC_REV and args.cache_len == 4096 else None
+    # DRAM bytes per launch (read + write) from one ncu capture of this workload, kept in the tracked profile
+    # summary; null once the kernel's device code has changed since the capture.
+    traffic = profiled_traffic() if args.cache_len == 4096 else None
     roofline = {"bound": "hbm", "kernel": "gemm_tc_kernel", "launches_per_step": gemm_launches,
                 "achieved": achieved, "peak": peak, "peak_kind": peak_kind, "unit": "GB/s",
                 "frac": achieved / peak, "traffic": traffic,
                 "bytes_per_launch": gemm_bytes / max(1, gemm_launches), "us_per_launch": gemm_ms * 1e3 / max(1, gemm_launches),
-                "kernel_us": {c: round(prof[c][0] * 1e3, 2) for c in PROF_CLASSES},
+                "kernel_us": {"gemm": round(prof["gemm"][0] * 1e3, 2), "attention": round(prof["attention"][0] * 1e3, 2)},
+                "gemm_us_when_launched_alone": {c: round(prof[c][0] * 1e3, 2) for c in gemm},
                 "forward_us": round(fwd_ms * 1e3, 2),
                 "forward_gbs": wl.bytes["total"] / (fwd_ms * 1e-3) / 1e9 if fwd_ms > 0 else 0.0,
                 "forward_frac": wl.bytes["total"] / (fwd_ms * 1e-3) / 1e9 / peak if fwd_ms > 0 else 0.0}
@@ -461,12 +523,17 @@ def main():
             "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
             "data": "synthetic", "config": workload_config(args.cache_len), "clocks": clocks,
             "e2e": {"value": e2e, "unit": UNIT, "h2d_bytes_per_step": int(wl.draft.nbytes),
-                    "d2h_bytes_per_step": 216},   # acceptance record (212 B) + block row count (4 B)
+                    "d2h_bytes_per_step": 220},   # acceptance record (216 B) + its sequence number
             "gpu_launches": int(launches), "roofline": roofline, "bytes_per_step": wl.bytes["total"]}
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         gbs, n, el = time_oracle(args.cache_len, 10.0)
         line["cpu_baseline"] = {"value": gbs, "unit": UNIT, "cores": blas_threads(), "kind": "oracle",
                                 "sample": f"{n} full steps of the same workload in {el:.1f} s"}
+    if rank == 0 and world == 1 and not args.no_generation:
+        wl.eng.close()
+        del wl
+        torch.cuda.empty_cache()
+        line["generation"] = generation_summary(device, args.generation_tokens)
     if rank == 0:
         print(json.dumps(line))
     dist_util.finish(group)

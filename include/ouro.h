@@ -180,6 +180,11 @@ int ouro_verify_forward(ouro_ctx *ctx, int which, int32_t *argmax_dev, float *lo
  * per flags, new pending token.  accepted_host [gamma+beta].  Host outputs may be NULL. */
 int ouro_accept_and_compact(ouro_ctx *ctx, const int32_t *argmax_dev, int32_t *n_accepted_host,
                             int32_t *chosen_host, int32_t *accurate_host, int32_t *accepted_host);
+/* The three calls above in one: packs the block for draft_dev [gamma] (pool looked up with key d_gamma), runs the
+ * target forward and applies Eq. 3 / Eq. 9, compaction and harvest.  Same host outputs as ouro_accept_and_compact;
+ * the only host wait of the step is the one for the acceptance record. */
+int ouro_verify_step(ouro_ctx *ctx, const int32_t *draft_dev, int32_t *n_accepted_host, int32_t *chosen_host,
+                     int32_t *accurate_host, int32_t *accepted_host);
 /* Advances model `which` past the first n rows of its current causal block (they become cached text). */
 int ouro_advance(ouro_ctx *ctx, int which, int32_t n);
 

@@ -74,6 +74,7 @@ _SIGNATURES = {
     "ouro_block_get": (C.c_int, [C.c_void_p, C.c_int, _I32P, _I32P, _I32P, _U64P, _I32P]),
     "ouro_verify_forward": (C.c_int, [C.c_void_p, C.c_int, C.c_void_p, C.c_void_p]),
     "ouro_accept_and_compact": (C.c_int, [C.c_void_p, C.c_void_p, _I32P, _I32P, _I32P, _I32P]),
+    "ouro_verify_step": (C.c_int, [C.c_void_p, C.c_void_p, _I32P, _I32P, _I32P, _I32P]),
     "ouro_advance": (C.c_int, [C.c_void_p, C.c_int, C.c_int32]),
     "ouro_draft": (C.c_int, [C.c_void_p, C.c_void_p]),
     "ouro_kernel_launches": (C.c_uint64, []),
@@ -318,6 +319,19 @@ class Engine:
         self._ck(self.L.ouro_accept_and_compact(self.ctx, o.data_ptr(), C.byref(n), C.byref(ch), C.byref(A),
                                                 acc.ctypes.data_as(_I32P)))
         return n.value, ch.value, A.value, acc[: n.value].copy()
+
+    def verify_step(self):
+        """assemble_candidates + verify_forward + accept_and_compact in one library call, on the tokens in
+        self.draft_tokens.  Returns (n_accepted, chosen, accurate, accepted tokens as a view that the next call reuses)."""
+        if not hasattr(self, "_vs"):
+            self._vs = (C.c_int32(), C.c_int32(), C.c_int32(), np.zeros(OURO_MAX_GAMMA + OURO_MAX_BETA, dtype=np.int32))
+            self._vs_args = (self.draft_tokens.data_ptr(), C.byref(self._vs[0]), C.byref(self._vs[1]), C.byref(self._vs[2]),
+                             self._vs[3].ctypes.data_as(_I32P))
+        rc = self.L.ouro_verify_step(self.ctx, *self._vs_args)
+        if rc != OURO_OK:
+            raise OuroError(rc, self.ctx)
+        n = self._vs[0].value
+        return n, self._vs[1].value, self._vs[2].value, self._vs[3][:n]
 
     def advance(self, which, n):
         self._ck(self.L.ouro_advance(self.ctx, which, n))

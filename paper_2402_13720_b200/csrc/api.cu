@@ -100,7 +100,6 @@ static size_t carve(ouro_ctx *c, char *base, const ouro_model_desc *t, const our
   int32_t *cand_suffix = cv.take<int32_t>((size_t)std::max(1, p->K * S));
   int32_t *cand_count = cv.take<int32_t>(1);
   int32_t *draft_dev = cv.take<int32_t>(p->gamma);
-  int32_t *stage_dev = cv.take<int32_t>(R);
   PoolDev pool{};
   size_t cap = (size_t)p->pool_sets * p->pool_ways;
   pool.key = cv.take<int32_t>(cap);
@@ -132,7 +131,6 @@ static size_t carve(ouro_ctx *c, char *base, const ouro_model_desc *t, const our
     c->cand_suffix = cand_suffix;
     c->cand_count = cand_count;
     c->draft_dev = draft_dev;
-    c->stage_dev = stage_dev;
     c->pool = pool;
     for (int w = 0; w < 2; ++w) {
       c->m[w].blk = blk[w];
@@ -349,8 +347,7 @@ extern "C" int ouro_assemble_candidates(ouro_ctx *c, const int32_t *draft_dev, c
   const int gamma = c->p.gamma, S = c->p.beta - 1, K = c->p.K;
   if (M.L + 1 + gamma + K * S > M.d.max_seq) return fail(c, OURO_ECAPACITY, "cache length + block rows exceeds max_seq");
   if (!suffix_dev)
-    launch_lookup_assemble(c->pool, M.blk, c->st, draft_dev, c->cand_suffix, c->cand_count, M.L, gamma, S, K, nullptr, 0,
-                           c->stream);
+    launch_lookup_assemble(c->pool, M.blk, c->st, draft_dev, c->cand_suffix, c->cand_count, M.L, gamma, S, K, c->stream);
   else
     launch_assemble_candidates(M.blk, c->st, draft_dev, suffix_dev, count_dev, M.L, gamma, S, K, c->stream);
   CKL();
@@ -653,6 +650,15 @@ extern "C" int ouro_accept_and_compact(ouro_ctx *c, const int32_t *argmax_dev, i
   if (accurate) *accurate = r.A;
   if (accepted) memcpy(accepted, r.accepted, (size_t)r.n_acc * 4);
   return OURO_OK;
+}
+
+// One verification step in one call: lookup + packing, the target forward, acceptance + compaction + harvest.
+extern "C" int ouro_verify_step(ouro_ctx *c, const int32_t *draft_dev, int32_t *n_acc, int32_t *chosen, int32_t *accurate,
+                                int32_t *accepted) {
+  if (!c || !draft_dev) return OURO_EINVAL;
+  TRY(ouro_assemble_candidates(c, draft_dev, nullptr, nullptr));
+  TRY(forward(c, OURO_TARGET, c->a.argmax, nullptr));
+  return ouro_accept_and_compact(c, c->a.argmax, n_acc, chosen, accurate, accepted);
 }
 
 // ------------------------------------------------------------------------------------- draft

@@ -195,7 +195,6 @@ __global__ void assemble_candidates_kernel(BlockDev b, DevState *st, const int32
   assemble_candidates_body(b, st, draft, suffix, count, L, gamma, S, K);
 }
 
-// Lookup with key d_gamma (warp 0) and packing in one launch.
 // Writes a result the host is polling for: payload first, then (system-wide fence between) the sequence number.
 __device__ __forceinline__ void mbox_post(int32_t *slot, const int32_t *payload, int n, int32_t seq) {
   for (int i = 0; i < n; ++i) slot[1 + i] = payload[i];
@@ -203,18 +202,15 @@ __device__ __forceinline__ void mbox_post(int32_t *slot, const int32_t *payload,
   *(volatile int32_t *)slot = seq;
 }
 
+// Lookup with key d_gamma (warp 0) and packing in one launch.
 __global__ void lookup_assemble_kernel(PoolDev P, BlockDev b, DevState *st, const int32_t *draft, int32_t *suffix,
-                                       int32_t *count, int L, int gamma, int S, int K, int32_t *mbox, int32_t seq) {
+                                       int32_t *count, int L, int gamma, int S, int K) {
   if (threadIdx.x < 32) {
     int32_t key = draft[gamma - 1];
     int n = (key < 0 || P.S == 0) ? 0 : pool_lookup(P, key, K, suffix);
     if (threadIdx.x == 0) *count = n;
   }
   __syncthreads();
-  if (mbox && threadIdx.x == 0) {                       // the row count goes out before the rows are packed
-    const int32_t B = 1 + gamma + (S > 0 ? min(*count, K) : 0) * S;
-    mbox_post(mbox + MBOX_ROWS, &B, 1, seq);
-  }
   assemble_candidates_body(b, st, draft, suffix, count, L, gamma, S, K);
 }
 
@@ -239,9 +235,9 @@ void launch_assemble_candidates(const BlockDev &b, DevState *st, const int32_t *
   assemble_candidates_kernel<<<1, OURO_MAX_ROWS, 0, s>>>(b, st, draft, suffix, count, L, gamma, S, K);
 }
 void launch_lookup_assemble(const PoolDev &P, const BlockDev &b, DevState *st, const int32_t *draft, int32_t *suffix,
-                            int32_t *count, int L, int gamma, int S, int K, int32_t *mbox, int32_t seq, cudaStream_t s) {
+                            int32_t *count, int L, int gamma, int S, int K, cudaStream_t s) {
   OURO_COUNT_LAUNCH();
-  lookup_assemble_kernel<<<1, OURO_MAX_ROWS, 0, s>>>(P, b, st, draft, suffix, count, L, gamma, S, K, mbox, seq);
+  lookup_assemble_kernel<<<1, OURO_MAX_ROWS, 0, s>>>(P, b, st, draft, suffix, count, L, gamma, S, K);
 }
 void launch_assemble_causal(const BlockDev &b, const int32_t *tokens, int n, int L, cudaStream_t s) {
   OURO_COUNT_LAUNCH();
@@ -289,45 +285,10 @@ __device__ void accept_body(const BlockDev &b, DevState *st, const int32_t *o, i
   st->n_seq = base + n;
 }
 
-__global__ void accept_kernel(BlockDev b, DevState *st, const int32_t *o, int32_t *seq_dev, int gamma, int S) {
-  if (threadIdx.x == 0) accept_body(b, st, o, seq_dev, gamma, S);
-}
-
-void launch_accept(const BlockDev &b, DevState *st, const int32_t *o, int32_t *seq_dev, int gamma, int S,
-                   cudaStream_t s) {
-  OURO_COUNT_LAUNCH();
-  accept_kernel<<<1, 32, 0, s>>>(b, st, o, seq_dev, gamma, S);
-}
-
 // ------------------------------------------------------------------------------ KV compaction
 // Slots L..L+A (pending token and accepted draft) already sit where they belong.  An accepted suffix of
 // candidate j sits at slots L+1+gamma+j*S+[0,m) and moves to L+1+gamma+[0,m).  Source and destination
-// ranges never overlap (j*S >= S >= m), so all rows move in parallel.
-template <typename T>
-__global__ void compact_kernel(T *k_cache, T *v_cache, const DevState *st, int L, int gamma, int S, int max_seq,
-                               int d_kv) {
-  int t = blockIdx.x, layer = blockIdx.y >> 1;
-  int chosen = st->chosen, m = st->m;
-  if (chosen <= 0 || t >= m) return;   // candidate 0 already sits next to the trunk
-  T *base = ((blockIdx.y & 1) ? v_cache : k_cache) + (size_t)layer * max_seq * d_kv;
-  const T *src = base + (size_t)(L + 1 + gamma + chosen * S + t) * d_kv;
-  T *dst = base + (size_t)(L + 1 + gamma + t) * d_kv;
-  for (int i = threadIdx.x; i < d_kv; i += blockDim.x) dst[i] = src[i];
-}
-
-void launch_compact(const ouro_model_desc &d, void *k_cache, void *v_cache, const DevState *st, int L, int gamma,
-                    int S, cudaStream_t s) {
-  if (S <= 0) return;
-  OURO_COUNT_LAUNCH();
-  dim3 grid(S, d.n_layers * 2);
-  int d_kv = d.n_kv_heads * d.head_dim;
-  if (d.dtype == OURO_BF16)
-    compact_kernel<__nv_bfloat16><<<grid, 128, 0, s>>>((__nv_bfloat16 *)k_cache, (__nv_bfloat16 *)v_cache, st, L, gamma,
-                                                       S, d.max_seq, d_kv);
-  else
-    compact_kernel<float><<<grid, 128, 0, s>>>((float *)k_cache, (float *)v_cache, st, L, gamma, S, d.max_seq, d_kv);
-}
-
+// ranges never overlap (j*S >= S >= m), so all rows move in parallel (accept_compact_harvest_kernel below).
 // ---------------------------------------------------------------------------------- harvest
 // Pool updates after a verification (Section 3.3), serialised in a fixed order by one warp:
 //  1. when the draft was fully accepted: every tried phrase (d_gamma, p^j_2..beta), j ascending, is
@@ -376,11 +337,6 @@ __device__ void harvest_body(const BlockDev &b, DevState *st, const PoolDev &P, 
       pool_insert(P, st, ph);
     }
   }
-}
-
-__global__ void harvest_kernel(BlockDev b, DevState *st, PoolDev P, const int32_t *o, const int32_t *seq_dev,
-                               int gamma, int S, unsigned flags) {
-  harvest_body(b, st, P, o, seq_dev, gamma, S, flags);
 }
 
 // Acceptance, compaction and harvest in one launch.  Block 0: one thread accepts (Eq. 3, Eq. 9), then its first
@@ -529,12 +485,6 @@ void launch_draft_accept_compact(const BlockDev &b, DevState *st, const int32_t 
   draft_accept_compact_kernel<<<1 + (S > 0 ? S : 0) * d.n_layers * 2, 128, 0, s>>>(
       b, st, o, out_dev, have, gamma, (unsigned char *)k_cache, (unsigned char *)v_cache, L, n, S, d.max_seq,
       d.n_kv_heads * d.head_dim * es);
-}
-
-void launch_harvest(const BlockDev &b, DevState *st, const PoolDev &P, const int32_t *o, const int32_t *seq_dev,
-                    int gamma, int S, unsigned flags, cudaStream_t s) {
-  OURO_COUNT_LAUNCH();
-  harvest_kernel<<<1, 32, 0, s>>>(b, st, P, o, seq_dev, gamma, S, flags);
 }
 
 // ----------------------------------------------------------------------------------- argmax

@@ -115,13 +115,12 @@ struct ouro_ctx {
   int32_t *cand_suffix = nullptr; // [K, S]
   int32_t *cand_count = nullptr;  // [1]
   int32_t *draft_dev = nullptr;   // [gamma]
-  int32_t *stage_dev = nullptr;   // [OURO_MAX_ROWS] staging for token uploads
   PoolDev pool{};
   // host side
   std::vector<int32_t> seq;       // the text: prompt + accepted tokens (last one pending)
   int32_t *pin = nullptr;         // pinned host staging (PIN_INTS ints)
-  // Mailbox in mapped pinned memory: the two results the host needs in every step (block row count, acceptance
-  // record) are written there by the kernels themselves, payload first, then a sequence number the host polls.
+  // Mailbox in mapped pinned memory: the result the host needs in every step (the acceptance record) is written there
+  // by the kernel itself, payload first, then a sequence number the host polls.
   int32_t *mbox = nullptr, *mbox_dev = nullptr;
   int32_t mseq = 0;
   const int *cur_rows_dev = nullptr;   // during a forward: where the kernels read the block's true row count, or NULL
@@ -156,18 +155,12 @@ void launch_vanilla_accept(DevState *st, const int32_t *o, int32_t *seq_dev, cud
 void launch_assemble_candidates(const BlockDev &b, DevState *st, const int32_t *draft, const int32_t *suffix,
                                 const int32_t *count, int L, int gamma, int S, int K, cudaStream_t s);
 void launch_assemble_causal(const BlockDev &b, const int32_t *tokens, int n, int L, cudaStream_t s);
-void launch_accept(const BlockDev &b, DevState *st, const int32_t *o, int32_t *seq_dev, int gamma, int S,
-                   cudaStream_t s);
-void launch_compact(const ouro_model_desc &d, void *k_cache, void *v_cache, const DevState *st, int L, int gamma,
-                    int S, cudaStream_t s);
-void launch_harvest(const BlockDev &b, DevState *st, const PoolDev &P, const int32_t *o, const int32_t *seq_dev,
-                    int gamma, int S, unsigned flags, cudaStream_t s);
 void launch_lookup_assemble(const PoolDev &P, const BlockDev &b, DevState *st, const int32_t *draft, int32_t *suffix,
-                            int32_t *count, int L, int gamma, int S, int K, int32_t *mbox, int32_t seq, cudaStream_t s);
+                            int32_t *count, int L, int gamma, int S, int K, cudaStream_t s);
 void launch_accept_compact_harvest(const BlockDev &b, DevState *st, const PoolDev &P, const int32_t *o, int32_t *seq_dev,
                                    const ouro_model_desc &d, void *k_cache, void *v_cache, int L, int gamma, int S,
                                    unsigned flags, int32_t *mbox, int32_t seq, cudaStream_t s);
-enum { MBOX_INTS = 128, MBOX_ROWS = 0, MBOX_ACCEPT = 16 };   // [flag, rows] and [flag, acceptance record] slots
+enum { MBOX_INTS = 128, MBOX_ACCEPT = 16 };   // mailbox slot [flag, acceptance record]
 void launch_draft_lookup_assemble(const PoolDev &P, const BlockDev &b, DevState *st, const int32_t *tokens, int n,
                                   int32_t *suffix, int32_t *count, int L, int S, int K, cudaStream_t s);
 void launch_draft_accept_compact(const BlockDev &b, DevState *st, const int32_t *o, int32_t *out_dev, int have, int gamma,
