@@ -17,6 +17,9 @@ What the paper fixes and what is this build's reading:
     sets x ways table addressed by the first token, LRU by a global stamp (PhrasePool below).
   * Phrase-level drafting on the draft model (Section 3.1) is not specified by the paper; PhraseDrafter
     is this build's reading: the draft model verifies pool phrases on itself, Section 3.2 style.
+  * Phrase generation during the draft forward (Section 3.1 defers to lookahead decoding) is not specified
+    either; LookaheadDrafter / window_phrases is this build's reading: a sliding window of guessed tokens
+    rides along every draft forward, one Jacobi step per forward, and its diagonals are the new phrases.
   * "Sub-segments of the discarded draft that match the verification" (Section 3.3) is read as
     in harvest_ops(); the replacement of tried phrases by their verified versions follows the
     second paragraph of Section 3.3.
@@ -27,7 +30,9 @@ causal forwards (Eq. 8); hand traces under tests/golden/; Eq. 3 / Eq. 9 / Eq. 10
 compaction equals a fresh prefill.  The pool policy and the harvest readings are this build's
 (the paper is silent); each is fixed by a hand-worked trace: the pool by its policy trace, the matched
 sub-segments and tried phrases by the three step traces, the two extensions (windows of the accepted
-text, windows of the prompt) by trace_harvest_accepted.txt and trace_seed_prompt.txt.
+text, windows of the prompt) by trace_harvest_accepted.txt and trace_seed_prompt.txt, the lookahead window's
+phrases by trace_window_phrases.txt; its block (positions, mask) by the Jacobi fixed point: a window that
+already holds the draft model's greedy continuation reproduces it.
 """
 from __future__ import annotations
 
@@ -331,6 +336,64 @@ class PhraseDrafter:
             c.length = L + n + mk
             out += gained[:keep]
             feed = [out[-1]]
+        return out
+
+    def rollback(self, valid_len):
+        self.cache.length = min(self.cache.length, valid_len)
+
+
+def window_phrases(src, chain, S):
+    """Phrases one draft forward with a lookahead window yields (this build's reading of Section 3.1's "multiple new
+    phrases are generated in parallel during each forward of the draft model"; the paper gives no procedure).
+
+    src[0] is the last real token the forward was fed and src[1..W] the window's guesses for the positions after
+    it; chain[i] is the draft model's greedy output at the row that holds src[i], i.e. its prediction for the next
+    position given the real text and the guesses src[1..i].  Along the diagonal, src[i] followed by chain[i],
+    chain[i+1], .., chain[i+S-1] is a beta-gram whose every token after the first is a draft-model prediction (exact
+    greedy text wherever the guesses before it were right).  One phrase per start i = 0 .. W-S+1, in that order."""
+    W = len(src) - 1
+    assert len(chain) == W + 1
+    return [tuple(int(t) for t in [src[i]] + list(chain[i:i + S])) for i in range(0, W - S + 2)] if S >= 1 else []
+
+
+class LookaheadDrafter:
+    """Token-level drafting (Eq. 1) in which every draft forward also carries a window of W guessed tokens for
+    the positions that follow, in the manner of the Jacobi iteration of lookahead decoding that Section 3.1 points to.
+
+    The block of a draft forward is the text the draft model has not cached yet followed by the window, packed like
+    one candidate suffix (Eq. 8 mask: window row i sees the text and window rows 1..i).  The real rows give the next
+    draft token exactly as in plain drafting (the window rows are invisible to them); the window rows give the
+    model's predictions under the guessed context.  Those predictions (a) become the next forward's guesses - the
+    window slides with the text, one Jacobi step per forward; a window that holds the draft model's own greedy
+    continuation is a fixed point - and (b) yield new phrases for the pool (window_phrases), inserted at once, so
+    that the verification that follows can already look them up.  Drafts are exactly those of ModelDrafter."""
+
+    def __init__(self, W, P, pool, width):
+        self.W, self.P, self.pool, self.width = W, P, pool, width
+        self.cache = tf.KVCache(W.desc)
+        self.window = None
+        self.calls = 0
+
+    def draft(self, seq, gamma, step):
+        c, S, out = self.cache, self.P.S, []
+        if self.window is None:       # first guesses: the text's own last tokens (any tokens would do)
+            tail = [int(t) for t in seq[-self.width:]] if self.width else []
+            self.window = [int(seq[-1])] * (self.width - len(tail)) + tail
+        feed = [int(t) for t in seq[c.length:]]
+        for _ in range(gamma):
+            n, L = len(feed), c.length
+            cands = [list(self.window)] if self.width else []
+            tokens, pos, group, visible = build_block(L, feed[0], feed[1:], cands)
+            o = tf.argmax_rows(tf.forward(self.W, c, tokens, pos, visible))
+            self.calls += 1
+            c.length = L + n                                     # the window's K/V rows are left behind
+            chain = [int(o[n - 1])] + [int(t) for t in o[n:n + self.width]]
+            if self.width:
+                for ph in window_phrases([feed[-1]] + self.window, chain, S):
+                    self.pool.insert(ph)
+                self.window = chain[1:]                          # predictions for the positions after the new token
+            feed = [chain[0]]
+            out.append(chain[0])
         return out
 
     def rollback(self, valid_len):

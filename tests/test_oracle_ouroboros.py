@@ -418,3 +418,72 @@ def test_draft_accept_planted_mistake():
     assert ob.draft_accept(tokens, o, n, S, 2) == (1, 3, [20, 30, 31, 55])
     assert ob.draft_accept(tokens, o, n, S, 1) == (0, 2, [20, 21, 99])
     assert ob.draft_accept(tokens, o, n, S, 0) == (-1, 0, [20])
+
+
+# ------------------------------------------------- phrase generation during the draft forward (Section 3.1)
+
+def test_hand_trace_window_phrases():
+    t = load_trace("trace_window_phrases.txt")
+    for beta in (3, 4, 5, 6, 7):
+        got = ob.window_phrases(t["src"], t["chain"], beta - 1)
+        assert [list(p) for p in got] == t[f"phrases_beta{beta}"]
+    assert t["chain"][1:] == t["next_window"]
+
+
+def test_lookahead_window_fixed_point_and_drafts(c1):
+    """Jacobi fixed point: a window that already holds the draft model's own greedy continuation is reproduced by the
+    forward (each window row then sees exactly the true text), which pins the window rows' positions and mask against
+    plain causal decoding; a wrong mask (window rows not seeing each other) fails it.  The drafts themselves are those
+    of the plain token-level drafter whatever the window holds."""
+    W, Wd = c1
+    P = C1P
+    width = 6
+    prompt = [int(t) for t in synth.prompt(7, C1T.vocab, 20, 0.0, 4, 4)]
+    cont = ob.vanilla_greedy(Wd, prompt, P.gamma + width + 2)            # the draft model's own greedy text
+    pool = ob.PhrasePool(P.pool_sets, P.pool_ways, P.beta)
+    d = ob.LookaheadDrafter(Wd, P, pool, width)
+    d.window = cont[:width]                                              # exact guesses for the positions after the prompt
+    out = d.draft(prompt, 1, 0)
+    assert out == cont[:1] and d.window == cont[1:1 + width]             # reproduced and slid by one
+    bad = ob.LookaheadDrafter(Wd, P, ob.PhrasePool(P.pool_sets, P.pool_ways, P.beta), width)
+    bad.window = cont[:width]
+    import unittest.mock as um
+    real_block = ob.build_block
+
+    def wrong_mask(L, pending, draft, cands):                            # window rows that do not see one another
+        tokens, pos, group, vis = real_block(L, pending, draft, cands)
+        n = 1 + len(draft)
+        for r in range(n, len(tokens)):
+            vis[r, L + n:L + r] = False
+        return tokens, pos, group, vis
+
+    with um.patch.object(ob, "build_block", wrong_mask):
+        bad.draft(prompt, 1, 0)
+    assert bad.window != cont[1:1 + width]
+    # every phrase of that forward is then exact greedy text of the draft model
+    text = prompt + cont
+    for _, ph in pool.export():
+        k = [i for i in range(len(prompt) - 1, len(text) - P.beta + 1) if tuple(text[i:i + P.beta]) == ph]
+        assert k, ph
+    # garbage guesses: the drafts are still those of plain drafting (the real rows never see the window)
+    d2 = ob.LookaheadDrafter(Wd, P, ob.PhrasePool(P.pool_sets, P.pool_ways, P.beta), width)
+    d2.window = [(cont[i] + 1) % C1T.vocab for i in range(width)]
+    assert d2.draft(prompt, P.gamma, 0) == ob.ModelDrafter(Wd).draft(prompt, P.gamma, 0) == cont[:P.gamma]
+    # width 0: nothing but plain drafting, the pool is not touched
+    p0 = ob.PhrasePool(P.pool_sets, P.pool_ways, P.beta)
+    d0 = ob.LookaheadDrafter(Wd, P, p0, 0)
+    assert d0.draft(prompt, P.gamma, 0) == cont[:P.gamma] and p0.export() == []
+
+
+@pytest.mark.parametrize("seed", [0, 4])
+def test_lossless_with_lookahead_drafter(c1, seed):
+    """Phrases made during drafting change what is verified, never the text (Eq. 4); with the target's own weights as
+    the draft model the window's phrases are the target's continuation and get accepted."""
+    W, Wd = c1
+    prompt = synth.prompt(seed, C1T.vocab, C1R["n"], C1R["copy_frac"], *C1R["span"])
+    ref = ob.vanilla_greedy(W, prompt, 40)
+    for draft_w in (Wd, W):
+        pool = ob.PhrasePool(C1P.pool_sets, C1P.pool_ways, C1P.beta)
+        out, stats = ob.generate(W, ob.LookaheadDrafter(draft_w, C1P, pool, 6), prompt, 40, C1P, pool=pool)
+        assert out == ref
+    assert sum(stats["m"]) > 0 and sum(stats["n_cand"]) > 0       # self-draft: suffixes from the window's phrases accepted
