@@ -43,7 +43,7 @@ enum {
 
 enum { OURO_F32 = 0, OURO_BF16 = 1 };
 enum { OURO_TARGET = 0, OURO_DRAFT = 1 };
-enum { OURO_MAX_ROWS = 128, OURO_MAX_BETA = 16, OURO_MAX_K = 16, OURO_MAX_GAMMA = 32 };
+enum { OURO_MAX_ROWS = 128, OURO_MAX_BETA = 16, OURO_MAX_K = 16, OURO_MAX_GAMMA = 32, OURO_MAX_WINDOW = 32 };
 
 /* ouro_params.flags */
 enum {
@@ -92,6 +92,9 @@ typedef struct {
   int32_t gamma, beta, K, pool_sets, pool_ways;
   uint32_t flags;
   int32_t eos_token;          /* < 0: none */
+  int32_t window;             /* Section 3.1, phrase generation during drafting: width W of the lookahead window that rides
+                                 along every forward of the draft model (see ouro_draft); 0: off.  <= OURO_MAX_WINDOW; not
+                                 together with OURO_DRAFT_PHRASES. */
 } ouro_params;
 
 typedef struct ouro_stats {
@@ -195,7 +198,14 @@ int ouro_advance(ouro_ctx *ctx, int which, int32_t n);
  * start with the last known token, go through one draft forward under the mask of Eq. 8; the draft model's
  * greedy outputs accept the longest matching phrase prefix (Eq. 9) and one more token, and its cache is
  * compacted like the target's.  The tokens are those of token-level drafting; only the number of draft
- * forwards (ouro_stats.draft_calls) changes.  The pool is read, not written, while drafting. */
+ * forwards (ouro_stats.draft_calls) changes.  The pool is read, not written, while drafting.
+ * With ouro_params.window = W > 0 (token-level drafting) every draft forward also carries W guessed tokens for the
+ * positions that follow, packed like one candidate suffix (Eq. 8 mask).  The paper says that new phrases are generated
+ * in parallel during each forward of the draft model and leaves the procedure to lookahead decoding; here the window
+ * rows' greedy outputs (a) become the next forward's guesses (the window slides with the text, one Jacobi step per
+ * forward) and (b) give beta-grams along the diagonal - a guess followed by the predictions after it - that enter the
+ * pool at once, W - beta + 3 per forward, so that the verification that follows can look them up.  The draft tokens are
+ * unchanged. */
 int ouro_draft(ouro_ctx *ctx, int32_t *draft_dev);
 
 /* Whole loops.  out_host [max_new]; *n_out tokens written (stops at eos_token).  ouro_generate is the

@@ -39,7 +39,7 @@ class ModelMemC(C.Structure):
 
 class ParamsC(C.Structure):
     _fields_ = [(n, C.c_int32) for n in ("gamma", "beta", "K", "pool_sets", "pool_ways")] + \
-               [("flags", C.c_uint32), ("eos_token", C.c_int32)]
+               [("flags", C.c_uint32), ("eos_token", C.c_int32), ("window", C.c_int32)]
 
 
 class StatsC(C.Structure):
@@ -133,7 +133,7 @@ def params_c(p: synth.DecodeParams) -> ParamsC:
     flags = (OURO_HARVEST_MATCHED if p.harvest_matched else 0) | (OURO_HARVEST_CANDIDATES if p.harvest_candidates else 0) | \
             (OURO_HARVEST_ACCEPTED if p.harvest_accepted else 0) | (OURO_SEED_PROMPT if p.seed_prompt else 0) | \
             (OURO_DRAFT_PHRASES if getattr(p, "draft_phrases", False) else 0)
-    return ParamsC(p.gamma, p.beta, p.K, p.pool_sets, p.pool_ways, flags, p.eos_token)
+    return ParamsC(p.gamma, p.beta, p.K, p.pool_sets, p.pool_ways, flags, p.eos_token, getattr(p, "window", 0))
 
 
 def lm_head_static(x: torch.Tensor, lm_head: torch.Tensor, want_logits: bool = False):

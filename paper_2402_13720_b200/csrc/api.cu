@@ -68,6 +68,7 @@ static bool params_ok(const ouro_params *p) {
   if (p->gamma < 1 || p->gamma > OURO_MAX_GAMMA || p->beta < 1 || p->beta > OURO_MAX_BETA) return false;
   if (p->K < 0 || p->K > OURO_MAX_K) return false;
   if (p->pool_sets < 1 || (p->pool_sets & (p->pool_sets - 1)) || p->pool_ways < 1) return false;
+  if (p->window < 0 || p->window > OURO_MAX_WINDOW || (p->window > 0 && (p->flags & OURO_DRAFT_PHRASES))) return false;
   return 1 + p->gamma + p->K * (p->beta - 1) <= OURO_MAX_ROWS;
 }
 
@@ -100,6 +101,7 @@ static size_t carve(ouro_ctx *c, char *base, const ouro_model_desc *t, const our
   int32_t *cand_suffix = cv.take<int32_t>((size_t)std::max(1, p->K * S));
   int32_t *cand_count = cv.take<int32_t>(1);
   int32_t *draft_dev = cv.take<int32_t>(p->gamma);
+  int32_t *win_dev = cv.take<int32_t>(OURO_MAX_WINDOW);
   PoolDev pool{};
   size_t cap = (size_t)p->pool_sets * p->pool_ways;
   pool.key = cv.take<int32_t>(cap);
@@ -131,6 +133,7 @@ static size_t carve(ouro_ctx *c, char *base, const ouro_model_desc *t, const our
     c->cand_suffix = cand_suffix;
     c->cand_count = cand_count;
     c->draft_dev = draft_dev;
+    c->win_dev = win_dev;
     c->pool = pool;
     for (int w = 0; w < 2; ++w) {
       c->m[w].blk = blk[w];
@@ -725,7 +728,30 @@ static int draft_step(ouro_ctx *c, int32_t *out_dev, int *calls) {
   }
   if (!D.present) return OURO_OK;
   if (!ext && (c->p.flags & OURO_DRAFT_PHRASES)) return draft_step_phrases(c, out_dev, calls);
-  if ((int)c->seq.size() + gamma > D.d.max_seq) return fail(c, OURO_ECAPACITY, "draft cache full");
+  if ((int)c->seq.size() + gamma + c->p.window > D.d.max_seq) return fail(c, OURO_ECAPACITY, "draft cache full");
+  if (c->p.window > 0) {
+    // Section 3.1, phrase generation during drafting (see ouro_draft in the header): every draft forward carries the
+    // lookahead window behind its text rows; its outputs refill the window and feed the pool, all on the device.
+    const int W = c->p.window, n_seq = (int)c->seq.size();
+    if (n_seq - D.L + W > OURO_MAX_ROWS) TRY(feed_text(c, OURO_DRAFT, n_seq - 1, nullptr));
+    for (int i = 0; i < gamma; ++i) {
+      const int n = i == 0 ? n_seq - D.L : 1;
+      if (n < 1) return fail(c, OURO_ESTATE, "draft cache ahead of the text");
+      launch_draft_window_assemble(D.blk, c->st, i == 0 ? c->seq_dev + D.L : out_dev + i - 1, n, c->win_dev, W, c->seq_dev,
+                                   D.L, c->stream);
+      D.blk_rows = n + W;
+      D.blk_rows_dev = false;
+      D.blk_L = D.L;
+      D.blk_is_candidate = true;
+      TRY(forward(c, OURO_DRAFT, c->a.argmax, nullptr));
+      launch_draft_window_harvest(D.blk, c->st, c->pool, c->a.argmax, ext ? nullptr : out_dev + i, n, W, c->win_dev, c->stream);
+      D.L += n;
+      D.blk_rows = 0;
+      *calls += 1;
+    }
+    CKL();
+    return OURO_OK;
+  }
   int last = 0;
   TRY(feed_text(c, OURO_DRAFT, (int)c->seq.size(), &last));
   *calls += 1;

@@ -487,6 +487,81 @@ void launch_draft_accept_compact(const BlockDev &b, DevState *st, const int32_t 
       d.n_kv_heads * d.head_dim * es);
 }
 
+// ------------------------------------------- phrase generation during the draft forward (Section 3.1)
+// A draft forward with a lookahead window: rows 0..n-1 are text the draft model is fed, rows n..n+W-1 hold the
+// window's guesses for the W positions that follow, packed like one candidate suffix (window row i sees the text and
+// window rows 1..i).  An empty window (after a reset) is first filled from the end of the text.
+__global__ void draft_window_assemble_kernel(BlockDev b, DevState *st, const int32_t *tokens, int n, int32_t *win, int W,
+                                             const int32_t *seq_dev, int L) {
+  const int r = threadIdx.x;
+  if (!st->win_valid) {
+    const int n_seq = st->n_seq;
+    if (r < W) {
+      const int src = n_seq - W + r;                      // the text's last W tokens; a short text repeats its last one in front
+      win[r] = seq_dev[src >= 0 ? src : n_seq - 1];
+    }
+  }
+  __syncthreads();
+  if (r == 0) {
+    st->win_valid = 1;
+    st->n_cand = W > 0 ? 1 : 0;
+    st->n_rows = n + W;
+  }
+  if (r >= n + W) return;
+  u64 m0 = 0, m1 = 0;
+  if (r < n) {
+    b.tok[r] = tokens[r];
+    b.pos[r] = L + r;
+    b.group[r] = 0;
+    b.lin_end[r] = L + r + 1;
+    b.seg_start[r] = 0;
+    b.seg_len[r] = 0;
+    for (int c = 0; c <= r; ++c) (c < 64 ? m0 : m1) |= 1ull << (c & 63);
+  } else {
+    const int i = r - n + 1;
+    b.tok[r] = win[i - 1];
+    b.pos[r] = L + n - 1 + i;
+    b.group[r] = 1;
+    b.lin_end[r] = L + n;
+    b.seg_start[r] = L + n;
+    b.seg_len[r] = i;
+    for (int c = 0; c <= r; ++c) (c < 64 ? m0 : m1) |= 1ull << (c & 63);
+  }
+  b.mask[2 * r] = m0;
+  b.mask[2 * r + 1] = m1;
+}
+
+// After that forward: chain[0] = o[n-1] is the next draft token; chain[i] = o[n-1+i] is the prediction after window
+// guess i.  The beta-grams along the diagonal, (src[i], chain[i], .., chain[i+S-1]) for i = 0 .. W-S+1 with src[0] the
+// last text token and src[i] guess i, enter the pool in that order; then the window becomes chain[1..W].
+__global__ void draft_window_harvest_kernel(BlockDev b, DevState *st, PoolDev P, const int32_t *o, int32_t *out, int n, int W,
+                                            int32_t *win) {
+  const int lane = threadIdx.x, S = P.S;
+  int32_t ph[OURO_MAX_BETA];
+  if (S >= 1)
+    for (int i = 0; i + S - 1 <= W; ++i) {
+      ph[0] = b.tok[n - 1 + i];
+      for (int q = 0; q < S; ++q) ph[1 + q] = o[n - 1 + i + q];
+      pool_insert(P, st, ph);
+    }
+  __syncwarp();
+  const int32_t next = lane < W ? o[n + lane] : 0;
+  __syncwarp();
+  if (lane < W) win[lane] = next;
+  if (lane == 0 && out) *out = o[n - 1];
+}
+
+void launch_draft_window_assemble(const BlockDev &b, DevState *st, const int32_t *tokens, int n, int32_t *win, int W,
+                                  const int32_t *seq_dev, int L, cudaStream_t s) {
+  OURO_COUNT_LAUNCH();
+  draft_window_assemble_kernel<<<1, OURO_MAX_ROWS, 0, s>>>(b, st, tokens, n, win, W, seq_dev, L);
+}
+void launch_draft_window_harvest(const BlockDev &b, DevState *st, const PoolDev &P, const int32_t *o, int32_t *out_or_null,
+                                 int n, int W, int32_t *win, cudaStream_t s) {
+  OURO_COUNT_LAUNCH();
+  draft_window_harvest_kernel<<<1, 32, 0, s>>>(b, st, P, o, out_or_null, n, W, win);
+}
+
 // ----------------------------------------------------------------------------------- argmax
 // Greedy choice per row; equal maxima resolve to the smallest token id.
 __global__ void argmax_kernel(const float *logits, int vocab, int32_t *out) {
@@ -555,6 +630,7 @@ __global__ void set_state_kernel(DevState *st, int32_t *seq_dev, int n_seq, int 
     st->n_cand = 0;
     st->n_rows = 0;
     st->status = 0;
+    st->win_valid = 0;
   }
 }
 void launch_set_state(DevState *st, int32_t *seq_dev, int n_seq, int pending, int fill, cudaStream_t s) {

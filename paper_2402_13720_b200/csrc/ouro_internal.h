@@ -56,6 +56,7 @@ struct DevState {
   // last phrase-level drafting round of the draft model (Section 3.1)
   int32_t d_keep;    // draft tokens the round added (at most what was still missing of gamma)
   int32_t d_cached;  // how many of them have their K/V in the draft cache (matched suffix tokens kept)
+  int32_t win_valid; // the lookahead window holds guesses (0 after a reset: the next draft forward fills it from the text)
 };
 
 // Per-row description of a query block.  Row r attends, in this order, cache slots [0, lin_end[r])
@@ -115,6 +116,7 @@ struct ouro_ctx {
   int32_t *cand_suffix = nullptr; // [K, S]
   int32_t *cand_count = nullptr;  // [1]
   int32_t *draft_dev = nullptr;   // [gamma]
+  int32_t *win_dev = nullptr;     // [OURO_MAX_WINDOW] lookahead window of the draft model
   PoolDev pool{};
   // host side
   std::vector<int32_t> seq;       // the text: prompt + accepted tokens (last one pending)
@@ -166,6 +168,10 @@ void launch_draft_lookup_assemble(const PoolDev &P, const BlockDev &b, DevState 
 void launch_draft_accept_compact(const BlockDev &b, DevState *st, const int32_t *o, int32_t *out_dev, int have, int gamma,
                                  const ouro_model_desc &d, void *k_cache, void *v_cache, int L, int n, int S,
                                  cudaStream_t s);
+void launch_draft_window_assemble(const BlockDev &b, DevState *st, const int32_t *tokens, int n, int32_t *win, int W,
+                                  const int32_t *seq_dev, int L, cudaStream_t s);
+void launch_draft_window_harvest(const BlockDev &b, DevState *st, const PoolDev &P, const int32_t *o, int32_t *out_or_null,
+                                 int n, int W, int32_t *win, cudaStream_t s);
 void launch_argmax(const float *logits, int rows, int vocab, int32_t *out, cudaStream_t s);
 void launch_pick_token(const int32_t *src, int index, int32_t *dst, cudaStream_t s);
 void launch_set_state(DevState *st, int32_t *seq_dev, int n_seq, int pending, int fill, cudaStream_t s);

@@ -126,6 +126,7 @@ class DecodeParams:
     harvest_accepted: bool = True     # beta-grams of the accepted text (extension, off in paper-pure mode)
     seed_prompt: bool = True          # beta-grams of the prompt (extension, off in paper-pure mode)
     draft_phrases: bool = False       # the draft model drafts phrase by phrase (Section 3.1)
+    window: int = 0                   # lookahead window riding along every draft forward (phrase generation, Section 3.1)
     eos_token: int = -1
 
     @property

@@ -850,3 +850,60 @@ def test_bounded_wait_gives_up_and_the_context_recovers():
     eng.set_drafter(None)
     assert len(van) == 12 and np.array_equal(out, van)
     eng.close()
+
+
+# ------------------------------------------------- phrase generation during the draft forward (Section 3.1)
+
+def test_lookahead_window_matches_oracle_c1():
+    """Every draft forward carries a lookahead window whose outputs refill it and feed the pool on the device: same text,
+    target calls, accepted suffix tokens and pool as the oracle's LookaheadDrafter; candidates come up and get accepted
+    without any phrase injected from outside."""
+    P = dataclasses.replace(C1P, window=6)
+    w = synth.model_weights(C1T, 0, device="cuda:0")
+    W = tf.Weights(C1T, synth.model_weights(C1T, 0))
+    for draft_desc in (C1D, C1T):                       # the early-exit draft, then the target as its own draft model
+        eng = binding.Engine(C1T, w, P, draft_desc, w)
+        Wd = tf.Weights(draft_desc, synth.model_weights(C1T, 0))
+        got_suffix = got_cand = 0
+        for seed in (1, 4):
+            prompt = synth.prompt(seed, C1T.vocab, C1R["n"], C1R["copy_frac"], *C1R["span"])
+            gen = C1R["gen"]
+            out, stats = eng.generate(prompt, gen)
+            pool_gpu = gpu_pool_rows(eng)
+            van, _ = eng.generate_vanilla(prompt, gen)
+            assert np.array_equal(out, van)
+            pool = oracle_pool(P)
+            drafter = ob.LookaheadDrafter(Wd, P, pool, P.window)
+            trace = []
+            ref, rstats = ob.generate(W, drafter, prompt, gen, P, pool=pool, trace=trace)
+            assert out.tolist() == ref
+            assert stats["target_calls"] == rstats["target_calls"] and stats["draft_calls"] == drafter.calls
+            assert stats["suffix_tokens"] == sum(rstats["m"]) and stats["candidates"] == sum(rstats["n_cand"])
+            assert pool_gpu[0] == [list(p) for _, p in trace[-1]["pool"]]
+            got_suffix += stats["suffix_tokens"]
+            got_cand += stats["candidates"]
+        assert got_cand > 0
+        if draft_desc is C1T:
+            assert got_suffix > 0                       # the window's phrases are the target's own continuation
+        eng.close()
+
+
+def test_lookahead_window_bf16_self_draft():
+    """The same on the tensor-core path (bf16, GQA, head dim 64): lossless, and the window's phrases extend accepted
+    drafts although nothing but the prompt and the draft model's own forwards feeds the pool."""
+    P0 = synth.DecodeParams(4, 9, 4, 32, 8)
+    P1 = dataclasses.replace(P0, window=10)
+    w = synth.model_weights(MIDB, 3, device="cuda:0")
+    prompt = synth.prompt(3, MIDB.vocab, 96, 0.3, 8, 32)
+    res = []
+    for P in (P0, P1):
+        eng = binding.Engine(MIDB, w, P, MIDB, w)
+        van, _ = eng.generate_vanilla(prompt, 120)
+        out, st = eng.generate(prompt, 120)
+        assert np.array_equal(out, van)
+        res.append(st)
+        eng.close()
+    assert res[1]["candidates"] > 0 and res[1]["suffix_tokens"] > 0
+    assert res[1]["target_calls"] <= res[0]["target_calls"]
+    with pytest.raises(binding.OuroError):              # a window together with phrase-level drafting is refused
+        binding.Engine(MIDB, w, dataclasses.replace(P1, draft_phrases=True), MIDB, w)
