@@ -317,6 +317,64 @@ def run_generate(args, device):
         "draft_forwards_per_target_call": st["draft_calls"] / st["target_calls"],
         "ms_draft_per_step": st["ms_draft"] / st["target_calls"], "identical_to_vanilla": bool(np.array_equal(out, van))}
     eng2.close()
+    # Phrase generation during the draft forward (Section 3.1): a lookahead window rides along every draft forward and
+    # feeds the pool on the device; nothing is injected from the host.  With a random-init pair the draft model's
+    # continuations rarely are the target's, so this run shows the cost of the window and whether candidates come up;
+    # the acceptance of such phrases is shown where the draft model is the target itself (tests, C1).
+    Pw = dataclasses.replace(P, window=max(P.S + 2, 12))
+    eng3 = binding.Engine(T, wt, Pw, D, wd, device=device)
+    out, st = eng3.generate(prompt, gen)
+    res["natural_lookahead_window"] = {
+        "window": Pw.window, "tokens_per_s": len(out) / (st["ms_total"] * 1e-3), "target_calls": st["target_calls"],
+        "candidates": st["candidates"], "suffix_tokens": st["suffix_tokens"],
+        "ms_draft_per_step": st["ms_draft"] / st["target_calls"], "identical_to_vanilla": bool(np.array_equal(out, van))}
+    # History reuse (Section 3.4): the same query again with the pool of the first run, and another query with it.
+    cold, stc = eng3.generate(prompt, gen)
+    warm, stw = eng3.generate(prompt, gen, keep_pool=True)
+    other = synth.prompt(SEED + 1, T.vocab, R["n"], R["copy_frac"], *R["span"])
+    o_cold, sto_c = eng3.generate(other, gen)
+    eng3.generate(prompt, gen)
+    o_warm, sto_w = eng3.generate(other, gen, keep_pool=True)
+    tps = lambda o, st_: round(len(o) / (st_["ms_total"] * 1e-3), 1)
+    res["history_reuse"] = {
+        "same_query": {"cold_tokens_per_s": tps(cold, stc), "warm_tokens_per_s": tps(warm, stw),
+                       "cold_target_calls": stc["target_calls"], "warm_target_calls": stw["target_calls"],
+                       "warm_suffix_tokens": stw["suffix_tokens"], "identical": bool(np.array_equal(cold, warm))},
+        "other_query": {"cold_tokens_per_s": tps(o_cold, sto_c), "warm_tokens_per_s": tps(o_warm, sto_w),
+                        "cold_target_calls": sto_c["target_calls"], "warm_target_calls": sto_w["target_calls"],
+                        "identical": bool(np.array_equal(o_cold, o_warm))}}
+    eng3.close()
+
+    # Algorithm 1 of the paper's Appendix B: coordinate search of gamma, W and beta on the wall-clock time of this
+    # generation (replayed drafts at the middle agreement level, the replayed phrase source, K = 3).
+    tuned = None
+    if args.tune:
+        from paper_2402_13720_b200 import tune
+
+        def clock(g, w_, b, k):
+            Pv = dataclasses.replace(P, gamma=g, window=w_, beta=b, K=k)
+            e4 = binding.Engine(T, wt, Pv, D, wd, device=device)
+
+            def drafter(seq, gg, step):
+                d = synth.corrupt_drafts(SEED + 7, truth, len(seq), gg, T.vocab, 0.12, 0.03, step)
+                grams = np.empty((Pv.K, Pv.beta), dtype=np.int32)
+                for j in range(Pv.K):
+                    grams[j, 0] = d[-1]
+                    grams[j, 1:] = synth.corrupt_drafts(SEED + 11 + j, truth, len(seq) + gg, Pv.S, T.vocab, 0.08 * (j + 1), 0.0, step)
+                e4.phrase_update(grams[::-1])
+                return d
+
+            e4.set_drafter(drafter)
+            o4, st4 = e4.generate(prompt, gen)
+            e4.set_drafter(None)
+            e4.close()
+            assert np.array_equal(o4, van)
+            return st4["ms_total"]
+
+        g0, w0, b0, k0, hist = tune.heuristic_search(clock, args.task)
+        tuned = {"task_type": args.task, "gamma": g0, "window": w0, "beta": b0, "K": k0,
+                 "tokens_per_s": round(gen / (min(h[4] for h in hist) * 1e-3), 1),
+                 "evaluations": [{"gamma": h[0], "window": h[1], "beta": h[2], "ms": round(h[4], 2)} for h in hist]}
 
     # Sweeps over the method's knobs (the paper's K study, its gamma / beta grid and its component ablation, on
     # synthetic inputs): replayed drafts at the middle agreement level plus the seeded phrase source, one engine
@@ -374,6 +432,8 @@ def run_generate(args, device):
             "results": res}
     if sweep:
         line["sweep"] = sweep
+    if tuned:
+        line["algorithm1"] = tuned
     print(json.dumps(line))
     eng.close()
 
@@ -440,6 +500,9 @@ def main():
                          "(vanilla greedy vs Ouroboros, natural and replayed drafts), one JSON line")
     ap.add_argument("--sweep", action="store_true", help="with --generate: K, gamma, beta and component sweeps as well")
     ap.add_argument("--gen-tokens", type=int, default=0, help="override the configuration's generation length")
+    ap.add_argument("--tune", action="store_true", help="with --generate: the paper's Algorithm 1 (coordinate search of "
+                    "gamma, W, beta on wall-clock time)")
+    ap.add_argument("--task", default="LH", choices=["HH", "LH"], help="recipe range of gamma for --tune")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
