@@ -301,30 +301,35 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_tc_kernel(const __grid_consta
     if (lane == 0) {
       // The weights do not depend on the previous kernel, so this warp never waits for it: the ring fills with
       // weight tiles while the predecessor drains.  The activation tiles come from warp 6, after its wait.
-      uint32_t n = 0;
+      // One thread runs this loop once per 16 KB stage; at 40 GB/s per SM that is every 0.4 us, so the loop carries
+      // no division and nothing that is constant over a span: stage index and ring round are counted along.
+      uint32_t n = 0, round = 0;
+      int st = 0;
       bool ok = true;
       for (int ci = 0; ci < cp.n && ok; ++ci) {
       const GemmParams &p = cp.g[ci];
-      auto issue = [&](const Span &s, int kb, int st) {
-        uint8_t *sa = ring + (size_t)st * stage_bytes;
-        mbar_expect_tx(&full[st], A_BYTES);
-        if (p.mode == MODE_SWIGLU) {
-          tma_load_2d(sa, &p.a[0], &full[st], kb * BLOCK_K, s.tile * 64, HINT_EVICT_FIRST);
-          tma_load_2d(sa + A_BYTES / 2, &p.a[1], &full[st], kb * BLOCK_K, s.tile * 64, HINT_EVICT_FIRST);
-        } else {
-          int seg, row0, col0, valid;
-          locate(p, s.tile, seg, row0, col0, valid);
-          tma_load_2d(sa, &p.a[seg], &full[st], kb * BLOCK_K, row0, HINT_EVICT_FIRST);
-        }
-      };
+      const bool swiglu = p.mode == MODE_SWIGLU;
       SpanWalker w(p);
       Span s;
       while (ok && w.next(s)) {
-        for (int kb = s.kb0; kb < s.kb1 && ok; ++kb, ++n) {
-          int st = n % n_stages;
-          if (n >= (uint32_t)n_stages) ok = mbar_wait(&empty[st], ((n / n_stages) - 1) & 1, abort_flag) && !*abort_flag;
-          if (!ok) break;
-          issue(s, kb, st);
+        int seg = 0, row0 = s.tile * 64, col0, valid;
+        if (!swiglu) locate(p, s.tile, seg, row0, col0, valid);
+        const CUtensorMap *m0 = &p.a[seg];
+        uint8_t *sa = ring + (size_t)st * stage_bytes;
+        for (int kb = s.kb0; kb < s.kb1; ++kb, ++n) {
+          if (round > 0) {
+            ok = mbar_wait(&empty[st], (round - 1) & 1, abort_flag) && !*abort_flag;
+            if (!ok) break;
+          }
+          mbar_expect_tx(&full[st], A_BYTES);
+          if (swiglu) {
+            tma_load_2d(sa, &p.a[0], &full[st], kb * BLOCK_K, row0, HINT_EVICT_FIRST);
+            tma_load_2d(sa + A_BYTES / 2, &p.a[1], &full[st], kb * BLOCK_K, row0, HINT_EVICT_FIRST);
+          } else {
+            tma_load_2d(sa, m0, &full[st], kb * BLOCK_K, row0, HINT_EVICT_FIRST);
+          }
+          sa += stage_bytes;
+          if (++st == n_stages) { st = 0; ++round; sa = ring; }
         }
       }
       TRACE(8);
@@ -336,7 +341,9 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_tc_kernel(const __grid_consta
     // ---------------------------------------------------------------- activation producer
     if (lane == 0) {
       pdl_wait();                                  // the first GEMM's activations are the previous kernel's output
-      uint32_t n = 0;
+      uint32_t n = 0, round = 0;
+      int st = 0;
+      uint8_t *sb = ring + A_BYTES;
       bool ok = true;
       if (cp.fold.part || cp.embed.table) {        // ... once every CTA has done its share of the fold / the gather
         ok = counter_wait(cp.finished + MAX_CHAIN, cp.fold_target, p0.status, 1u << 22);
@@ -355,12 +362,15 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_tc_kernel(const __grid_consta
         SpanWalker w(p);
         Span s;
         while (ok && w.next(s)) {
-          for (int kb = s.kb0; kb < s.kb1 && ok; ++kb, ++n) {
-            int st = n % n_stages;
-            if (n >= (uint32_t)n_stages) ok = mbar_wait(&empty[st], ((n / n_stages) - 1) & 1, abort_flag) && !*abort_flag;
-            if (!ok) break;
+          for (int kb = s.kb0; kb < s.kb1; ++kb, ++n) {
+            if (round > 0) {
+              ok = mbar_wait(&empty[st], (round - 1) & 1, abort_flag) && !*abort_flag;
+              if (!ok) break;
+            }
             mbar_expect_tx(&full[st], b_bytes);
-            tma_load_2d(ring + (size_t)st * stage_bytes + A_BYTES, &p.b, &full[st], kb * BLOCK_K, 0, HINT_EVICT_LAST);
+            tma_load_2d(sb, &p.b, &full[st], kb * BLOCK_K, 0, HINT_EVICT_LAST);
+            sb += stage_bytes;
+            if (++st == n_stages) { st = 0; ++round; sb = ring + A_BYTES; }
           }
         }
       }
@@ -371,7 +381,10 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_tc_kernel(const __grid_consta
     // ---------------------------------------------------------------- MMA issuer
     if (lane == 0) {
       const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(p0.t_pad >> 3) << 17) | ((uint32_t)(TILE_N >> 4) << 24);
-      uint32_t n = 0, item = 0;
+      uint32_t n = 0, item = 0, round = 0;
+      int st = 0;
+      uint32_t sa = smem_u32(ring);
+      const uint32_t ring0 = sa;
       bool ok = true;
       for (int ci = 0; ci < cp.n && ok; ++ci) {
       const GemmParams &p = cp.g[ci];
@@ -385,16 +398,16 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_tc_kernel(const __grid_consta
         fence_after_sync();
         uint32_t tmem_d = tmem_base + a * acc_cols;
         for (int kb = s.kb0; kb < s.kb1; ++kb, ++n) {
-          int st = n % n_stages;
-          ok = mbar_wait(&full[st], (n / n_stages) & 1, abort_flag) && !*abort_flag;
+          ok = mbar_wait(&full[st], round & 1, abort_flag) && !*abort_flag;
           if (!ok) break;
           if (first) { TRACE(2); first = false; }
           fence_after_sync();
-          uint32_t sa = smem_u32(ring + (size_t)st * stage_bytes), sb = sa + A_BYTES;
-          uint64_t da = smem_desc_sw128(sa), db = smem_desc_sw128(sb);
+          const uint64_t da = smem_desc_sw128(sa), db = smem_desc_sw128(sa + A_BYTES);
 #pragma unroll
           for (int k = 0; k < BLOCK_K / 16; ++k) mma_bf16(tmem_d, da + 2 * k, db + 2 * k, idesc, (kb > s.kb0 || k > 0) ? 1u : 0u);
           mma_commit(&empty[st]);
+          sa += stage_bytes;
+          if (++st == n_stages) { st = 0; ++round; sa = ring0; }
         }
         if (!ok) break;
         mma_commit(&acc_full[a]);
