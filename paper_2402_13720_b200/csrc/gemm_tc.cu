@@ -31,7 +31,7 @@ void ouro_set_global_error(const std::string &msg);   // api.cu
 // threads of every CTA stamp the global nanosecond timer at fixed points; ouro_trace_read_gemm copies the stamps
 // of the most recent launch of every kind out.  Compiled out by default.
 #ifdef OURO_TRACE
-__device__ unsigned long long g_gemm_trace[8][160][12];
+__device__ unsigned long long g_gemm_trace[8][160][16];
 __device__ __forceinline__ unsigned long long trace_now() {
   unsigned long long t;
   asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t)::"memory");
@@ -575,6 +575,10 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_tc_kernel(const __grid_consta
                 acc[j].x += tmp[cc][j].x; acc[j].y += tmp[cc][j].y; acc[j].z += tmp[cc][j].z; acc[j].w += tmp[cc][j].w;
               }
           }
+        }
+        if (!stg && tb == tb0 && gi == 0 && grp == 0) {
+          if (acc[0].x == 1.2345e-30f) TRACE(14);                    // (keeps the partial sums live up to here)
+          TRACE(12);
         }
         if (res_norm) {
           // new residual stream, its bf16(gain * x) image for the next GEMM, and this tile's sums of squares

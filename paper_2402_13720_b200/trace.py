@@ -54,10 +54,10 @@ def main():
         eng.verify_forward()
     torch.cuda.synchronize()
     lib = binding.lib()
-    g = (C.c_ulonglong * (8 * 160 * 12))()
+    g = (C.c_ulonglong * (8 * 160 * 16))()
     a = (C.c_ulonglong * (512 * 8))()
     assert lib.ouro_trace_read_gemm(g) == 0 and lib.ouro_trace_read_attn(a) == 0
-    g = np.array(g[:], dtype=np.int64).reshape(8, 160, 12)
+    g = np.array(g[:], dtype=np.int64).reshape(8, 160, 16)
     a = np.array(a[:], dtype=np.int64).reshape(512, 8)
 
     def stats(x):
@@ -66,7 +66,7 @@ def main():
     names = ["q,k,v", "o-proj", "gate,up", "down", "LM head"]
     points = [(0, "CTA entry"), (8, "last weight load issued"), (2, "first stage full"), (3, "last MMA issued"),
               (4, "last accumulator complete"), (5, "whole tiles done / fix-up begins"), (6, "partials of the others there"),
-              (9, "  group 0: past the wait + fence"), (10, "  group 0: its tokens finished"), (11, "  group 0: tile re-armed"),
+              (9, "  group 0: past the wait + fence"), (12, "  group 0: first batch added up"), (10, "  group 0: its tokens finished"), (11, "  group 0: tile re-armed"),
               (7, "fix-up done")]
     spans = []
     for kind in range(5):
