@@ -99,6 +99,8 @@ struct TmParams {
   int direct;                      // every row's keys lie in span 0: normalise and write `out`, no folding needed
   int *status;
   const int *rows_dev;             // NULL, or the block's true row count in device memory (`rows` is then an upper bound)
+  const uint8_t *pf_ptr[3];        // regions to bring into L2 for the kernels that follow (see L2Prefetch); each CTA asks
+  uint32_t pf_bytes[3];            // for an equal share of every region
 };
 
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -132,10 +134,12 @@ __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, Misc *
   if (atomicExch(&ms->abort_flag, 1) == 0) atomicExch(status, 1);
   return false;
 }
+// The cache rows are read once per forward pass: marked evict-first in L2, so that they do not push out the weights
+// prefetched for the kernels that follow.
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, uint64_t *bar, int x, int y) {
   asm volatile(
-      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];" ::"r"(dst),
-      "l"(map), "r"(smem_u32(bar)), "r"(x), "r"(y)
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%3, %4}], [%2], %5;" ::"r"(dst),
+      "l"(map), "r"(smem_u32(bar)), "r"(x), "r"(y), "l"(0x12F0000000000000ull)
       : "memory");
 }
 // K-major operand in 128-byte swizzle: rows of 128 bytes, 8-row groups 1024 bytes apart.
@@ -213,6 +217,18 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tm_kernel(const __grid_consta
   const int g = p.H / p.Hkv, dkv = p.Hkv * HD, M_all = g * rows, span0 = sc * SPAN;
 
   if (tid == 0) TRACE(0);
+  if (tid == 32) {
+    // the weights the next kernels start with do not depend on anything computed here: ask for this CTA's share now
+    const uint32_t u = blockIdx.y * gridDim.x + blockIdx.x, U = gridDim.x * gridDim.y;
+#pragma unroll
+    for (int r = 0; r < 3; ++r) {
+      const uint32_t bytes = p.pf_bytes[r];
+      if (bytes == 0) continue;
+      const uint32_t share = ((bytes + U - 1) / U + 15u) & ~15u, off = u * share;
+      if (off < bytes)
+        asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(p.pf_ptr[r] + off), "r"(min(share, bytes - off)) : "memory");
+    }
+  }
   if (sm_u & 1023) {                                   // the swizzled tiles need a 1024-byte aligned base
     if (tid == 0) atomicExch(p.status, 1);
     return;
@@ -650,9 +666,14 @@ int attention_tm_setup() {
 // that consumes the attention output); with a single span the kernel has written `out` itself.
 bool launch_attention_tm(const ouro_model_desc &d, const void *q, const void *kmap, const void *vmap, const void *k_cache,
                          const void *v_cache, const BlockDev &b, int rows, int L, int n_vis_max, int layer, float *part,
-                         void *out, int *status, const int *rows_dev, cudaStream_t s) {
+                         void *out, int *status, const int *rows_dev, const L2Prefetch &pf, cudaStream_t s) {
   OURO_COUNT_LAUNCH();
   TmParams p;
+  for (int r = 0; r < 3; ++r) {
+    const bool ok = pf.ptr[r] && pf.bytes[r] > 0 && pf.bytes[r] < (1ull << 31) && pf.bytes[r] % 16 == 0 && ((uintptr_t)pf.ptr[r] & 15) == 0;
+    p.pf_ptr[r] = ok ? (const uint8_t *)pf.ptr[r] : nullptr;
+    p.pf_bytes[r] = ok ? (uint32_t)pf.bytes[r] : 0u;
+  }
   p.kmap = *reinterpret_cast<const CUtensorMap *>(kmap);
   p.vmap = *reinterpret_cast<const CUtensorMap *>(vmap);
   size_t off = (size_t)layer * d.max_seq * d.n_kv_heads * d.head_dim;

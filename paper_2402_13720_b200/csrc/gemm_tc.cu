@@ -959,6 +959,7 @@ struct FastState {
   ChainParams chain{};          // GEMMs collected for the next launch
   int chain_kind[MAX_CHAIN] = {0, 0, 0, 0};
   bool fuse = true;             // run consecutive GEMMs as one launch
+  long pf_ffn_rows = 0;         // rows of gate and of up the attention kernel prefetches into L2 besides the output projection (< 0: nothing)
   bool dirty = false;           // a bounded wait gave up: counters must be cleared before the next launch
   uint32_t wait_limit = 1u << 22;   // polls of a partial-tile wait (ouro_debug_set_wait_limit)
 };
@@ -1022,6 +1023,8 @@ int ouro_fast_setup(ouro_ctx *c) {
   {
     const char *e = getenv("OURO_FUSE");                       // OURO_FUSE=0: every GEMM is a launch of its own
     f->s.fuse = !(e && e[0] == '0');
+    const char *pf = getenv("OURO_PF_ROWS");
+    if (pf) f->s.pf_ffn_rows = atol(pf);
   }
   f->s.tile_max = (float *)((char *)c->a.scratch + slots_bytes() + 2 * MAX_TILES * sizeof(int) + SPARE_BYTES);
   f->s.tile_arg = (int *)((char *)f->s.tile_max + tile_best_bytes());
@@ -1266,9 +1269,18 @@ int ouro_fast_layer(ouro_ctx *c, int which, int l, int rows) {
   {
     ProfScope ps(c, OURO_PROF_ATTENTION);
     bool pieces = false;             // the attention output is still in per-span pieces
-    if (c->fast->s.m[which].kv_maps)
+    if (c->fast->s.m[which].kv_maps) {
+      // what the launch after the attention streams first: the output projection, then the first rows of gate and up
+      L2Prefetch pf;
+      const size_t row_bytes = (size_t)d.d_model * 2, head = std::min<size_t>((size_t)d.d_ffn, c->fast->s.pf_ffn_rows) * row_bytes;
+      if (c->fast->s.pf_ffn_rows >= 0) {
+        pf.ptr[0] = M.wo[l]; pf.bytes[0] = (size_t)d.d_model * dq * 2;
+        pf.ptr[1] = M.w_gate[l]; pf.bytes[1] = head;
+        pf.ptr[2] = M.w_up[l]; pf.bytes[2] = head;
+      }
       pieces = launch_attention_tm(d, a.q, &c->fast->s.m[which].kmap, &c->fast->s.m[which].vmap, M.k_cache, M.v_cache, M.blk, rows,
-                                   M.L, M.L + rows, l, c->fast->s.attn_part, a.att, &c->st->status, c->cur_rows_dev, s);
+                                   M.L, M.L + rows, l, c->fast->s.attn_part, a.att, &c->st->status, c->cur_rows_dev, pf, s);
+    }
     else if (attention_tc_supported(d))
       pieces = launch_attention_tc(d, a.q, M.k_cache, M.v_cache, M.blk, rows, M.L, M.L + rows, l, c->fast->s.attn_part, a.att,
                                    c->cur_rows_dev, s);

@@ -207,6 +207,13 @@ bool launch_attention_tc(const ouro_model_desc &d, const void *q, const void *k_
 // ---- attn_tm.cu (tcgen05 path, head dim 128) ---------------------------------------------------
 bool attention_tm_supported(const ouro_model_desc &d);
 int attention_tm_setup();
+// Weights the kernels after the attention stream first (the output projection, the head of the gate and up matrices):
+// the attention kernel leaves most of the HBM bandwidth unused, so its CTAs ask for these bytes to be brought into L2
+// meanwhile.  Every region is a multiple of 16 bytes at a 16-byte aligned address; bytes 0 = no region.
+struct L2Prefetch {
+  const void *ptr[3] = {nullptr, nullptr, nullptr};
+  size_t bytes[3] = {0, 0, 0};
+};
 bool launch_attention_tm(const ouro_model_desc &d, const void *q, const void *kmap, const void *vmap, const void *k_cache,
                          const void *v_cache, const BlockDev &b, int rows, int L, int n_vis_max, int layer, float *part,
-                         void *out, int *status, const int *rows_dev, cudaStream_t s);
+                         void *out, int *status, const int *rows_dev, const L2Prefetch &pf, cudaStream_t s);
