@@ -21,6 +21,22 @@
 // a token gets bit-identical attention whether it is verified inside a candidate block or decoded alone.
 #include "ouro_internal.h"
 
+// Optional timeline (compile with -DOURO_TRACE): see gemm_tc.cu.
+#ifdef OURO_TRACE
+__device__ unsigned long long g_attn_tc_trace[512][8];
+__device__ __forceinline__ unsigned long long attn_tc_trace_now() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t)::"memory");
+  return t;
+}
+#define TRACE(slot) do { const int cta_ = (blockIdx.z * gridDim.y + blockIdx.y) * gridDim.x + blockIdx.x; if (threadIdx.x == 0 && cta_ < 512) g_attn_tc_trace[cta_][slot] = attn_tc_trace_now(); } while (0)
+extern "C" int ouro_trace_read_attn_tc(unsigned long long *out_host) {
+  return (int)cudaMemcpyFromSymbol(out_host, g_attn_tc_trace, sizeof(g_attn_tc_trace));
+}
+#else
+#define TRACE(slot) do { } while (0)
+#endif
+
 namespace {
 
 constexpr int CH = 128;            // keys per chunk
@@ -29,8 +45,11 @@ constexpr int SPAN = CH * SC;
 constexpr int WARPS = 8;
 constexpr int KW = CH / WARPS;     // keys per warp in the S phase (two 8-key MMA tiles)
 constexpr int THREADS = WARPS * 32;
-constexpr int QR = 64;             // query rows per round (4 MMA row tiles)
-constexpr int MT = QR / 16;
+// Query rows per round: MT row tiles of 16 (MT = 4: 64 rows, or MT = 1: 16 rows for short blocks such as a draft
+// model's single-row steps).  The kernel's loops over row tiles are unrolled, and with four tiles its machine code is
+// 150 KB, of which a block with one live tile still walks most: a pass over a chunk then takes 4.3 us waiting for
+// instruction fetches.  A row's arithmetic does not involve its tile's index or the other rows, so both sizes give the
+// same bits.
 
 struct AttnParams {
   const __nv_bfloat16 *q;          // [rows][H*HD] rotated queries
@@ -90,8 +109,9 @@ __device__ __forceinline__ void map_row(int m, int g, int rows, const int *grp, 
   }
 }
 
-template <int HD>
+template <int HD, int MT>
 struct Smem {
+  static constexpr int QR = 16 * MT;
   static constexpr int ROWB = HD * 2;                              // bytes per K/V/Q tile row
   static constexpr int KV = CH * ROWB;                             // one K or V buffer
   static constexpr int OFF_V = 2 * KV;                             // K[2] then V[2]
@@ -105,9 +125,10 @@ struct Smem {
   static constexpr int BYTES = OFF_MAP + QR * 4;
 };
 
-template <int HD>
+template <int HD, int MT>
 __global__ void __launch_bounds__(THREADS) attn_span_kernel(const AttnParams p) {
-  using S = Smem<HD>;
+  using S = Smem<HD, MT>;
+  constexpr int QR = S::QR;
   constexpr int CPR = HD / 8;                  // 16-byte pieces per row
   constexpr int ROWB = S::ROWB;
   constexpr int PW = HD + 2;
@@ -119,6 +140,7 @@ __global__ void __launch_bounds__(THREADS) attn_span_kernel(const AttnParams p) 
   const uint32_t sm_u = smem_u32(smem);
 
   pdl_trigger();
+  TRACE(0);
   // Everything up to pdl_wait() reads only what was complete before the forward pass began: the block description
   // (written by the assembling kernel, which is not launched programmatically and so has finished) and cache rows
   // below the cache length.  The queries and the block's own K/V rows come from the kernel just before this one.
@@ -186,7 +208,9 @@ __global__ void __launch_bounds__(THREADS) attn_span_kernel(const AttnParams p) 
     const int n_mt = (min(QR, M_all - m0) + 15) >> 4;  // row tiles that hold query rows; the others are skipped
 
     stage_common(0, 0);                                 // chunk 0 (its rows below the cache length) is on its way ...
+    TRACE(1);
     pdl_wait();                                         // ... while the previous kernel finishes
+    TRACE(2);
     for (int idx = threadIdx.x; idx < QR * CPR; idx += THREADS) {
       int row = idx / CPR, ch = idx % CPR, m = m0 + row;
       uint32_t off = S::OFF_Q + row * ROWB + ((ch ^ (row & 7)) << 4);
@@ -209,6 +233,7 @@ __global__ void __launch_bounds__(THREADS) attn_span_kernel(const AttnParams p) 
       const int buf = ci & 1, c0 = span0 + ci * CH;
       if (ci + 1 < n_chunks) { stage_common(ci + 1, buf ^ 1); cp_wait_but_one(); } else { cp_wait_all(); }
       __syncthreads();
+      if (ci == 0) TRACE(3);
       const bool common = c0 + CH <= p.L;
       int g_begin = 0;
       while (g_begin < rows) {
@@ -369,6 +394,7 @@ __global__ void __launch_bounds__(THREADS) attn_span_kernel(const AttnParams p) 
         g_begin = g_end;
       }
     }
+    TRACE(4);
     // ---- the span's piece of every row of the round that reaches it
 #pragma unroll
     for (int i = 0; i < 2 * MT; ++i) {
@@ -392,6 +418,7 @@ __global__ void __launch_bounds__(THREADS) attn_span_kernel(const AttnParams p) 
         *reinterpret_cast<float2 *>(dst + 2 + d) = make_float2(o[i >> 1][nt][2 * (i & 1)], o[i >> 1][nt][2 * (i & 1) + 1]);
       }
     }
+    TRACE(5);
   }
 }
 
@@ -407,12 +434,12 @@ size_t attention_tc_scratch_bytes(const ouro_model_desc &d) {
   return (size_t)OURO_MAX_ROWS * d.n_heads * cap * (d.head_dim + 2) * sizeof(float);
 }
 
+template <int HD, int MT>
+static bool tc_prepare() {
+  return cudaFuncSetAttribute(attn_span_kernel<HD, MT>, cudaFuncAttributeMaxDynamicSharedMemorySize, Smem<HD, MT>::BYTES) == cudaSuccess;
+}
 int attention_tc_setup() {
-  if (cudaFuncSetAttribute(attn_span_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, Smem<128>::BYTES) != cudaSuccess)
-    return OURO_ECUDA;
-  if (cudaFuncSetAttribute(attn_span_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, Smem<64>::BYTES) != cudaSuccess)
-    return OURO_ECUDA;
-  return OURO_OK;
+  return tc_prepare<128, 4>() && tc_prepare<128, 1>() && tc_prepare<64, 4>() && tc_prepare<64, 1>() ? OURO_OK : OURO_ECUDA;
 }
 
 // n_vis_max: an upper bound of the number of keys any row of the block sees (cache length + rows).
@@ -432,9 +459,15 @@ bool launch_attention_tc(const ouro_model_desc &d, const void *q, const void *k_
   p.part = part;
   p.out = (__nv_bfloat16 *)out;
   const int m_all = (d.n_heads / d.n_kv_heads) * rows;      // query rows per kv head, served 64 per CTA
-  dim3 grid((n_vis_max + SPAN - 1) / SPAN, d.n_kv_heads, (m_all + QR - 1) / QR);
+  const int mt = m_all <= 16 ? 1 : 4, qr = 16 * mt;         // rows per round (m_all is an upper bound when the count is on the device)
+  dim3 grid((n_vis_max + SPAN - 1) / SPAN, d.n_kv_heads, (m_all + qr - 1) / qr);
   p.direct = n_vis_max <= SPAN;                             // a single span: nothing to fold
-  if (d.head_dim == 128) launch_pdl(attn_span_kernel<128>, grid, THREADS, Smem<128>::BYTES, s, p);
-  else launch_pdl(attn_span_kernel<64>, grid, THREADS, Smem<64>::BYTES, s, p);
+  if (d.head_dim == 128) {
+    if (mt == 1) launch_pdl(attn_span_kernel<128, 1>, grid, THREADS, Smem<128, 1>::BYTES, s, p);
+    else launch_pdl(attn_span_kernel<128, 4>, grid, THREADS, Smem<128, 4>::BYTES, s, p);
+  } else {
+    if (mt == 1) launch_pdl(attn_span_kernel<64, 1>, grid, THREADS, Smem<64, 1>::BYTES, s, p);
+    else launch_pdl(attn_span_kernel<64, 4>, grid, THREADS, Smem<64, 4>::BYTES, s, p);
+  }
   return !p.direct;
 }

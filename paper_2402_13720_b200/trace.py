@@ -59,6 +59,8 @@ def main():
     assert lib.ouro_trace_read_gemm(g) == 0 and lib.ouro_trace_read_attn(a) == 0
     g = np.array(g[:], dtype=np.int64).reshape(8, 160, 16)
     a = np.array(a[:], dtype=np.int64).reshape(512, 8)
+    if not (a[:, 0] > 0).any():                  # head dim 64: the mma.sync attention kernel keeps a timeline of its own
+        assert lib.ouro_trace_read_attn_tc(a.ctypes.data_as(C.POINTER(C.c_ulonglong))) == 0
 
     def stats(x):
         return "min %6.1f  med %6.1f  max %6.1f" % (x.min(), np.median(x), x.max()) if len(x) else "-"
@@ -86,7 +88,7 @@ def main():
         t = a[live]
         t0 = t[:, 2].min()
         print(f"attention  ({live.sum()} CTAs)")
-        for col, nm in [(0, "CTA entry"), (1, "set-up done, waiting"), (2, "dependency wait over"), (3, "first scores"),
+        for col, nm in [(0, "CTA entry"), (1, "set-up done, waiting"), (2, "dependency wait over"), (3, "first scores"), (6, "(head dim 64) second chunk begins"), (7, "(head dim 64) third chunk begins"),
                         (4, "last pass accumulated"), (5, "CTA done")]:
             x = t[:, col][t[:, col] > 0]
             print("   %-34s %s" % (nm, stats((x - t0) / 1e3)))
