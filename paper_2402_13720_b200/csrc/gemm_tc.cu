@@ -503,7 +503,9 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_tc_kernel(const __grid_consta
       locate(p, tile, seg, row0, col0, valid);
       const int ng = gi & 31, tg = gi >> 5, TG = G >> 5;
       const int col = col0 + 4 * ng;
-      const bool full4 = 4 * ng + 3 < valid;
+      // Every matrix has a multiple of 8 output features (the shape checks see to it), so a thread's four columns are
+      // inside the matrix together or not at all.
+      const bool full4 = 4 * ng < valid;
       const int js = n * TG;                                         // token step inside a batch of four
       const int cm = row0 + 4 * ng;                                  // first of this thread's 4 columns inside q, k or v
       const int half = p.head_dim >> 1;
@@ -513,7 +515,7 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_tc_kernel(const __grid_consta
       float gn[4] = {0.f, 0.f, 0.f, 0.f};
       if (res_norm) {
 #pragma unroll
-        for (int e = 0; e < 4; ++e) gn[e] = 4 * ng + e < valid ? __bfloat162float(p.gain[col + e]) : 0.f;
+        for (int e = 0; e < 4; ++e) gn[e] = full4 ? __bfloat162float(p.gain[col + e]) : 0.f;
       }
       // what the epilogue reads besides the accumulators, for the four tokens of a batch at once
       auto load_ops = [&](int tb, float4 *oa, float4 *ob) {
@@ -524,13 +526,7 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_tc_kernel(const __grid_consta
           if (t >= t_lim) continue;
           if (res_norm) {
             const float *y = p.out_f32 + (size_t)t * p.ldo + col;
-            if (full4) {
-              oa[j] = *reinterpret_cast<const float4 *>(y);
-            } else {
-              if (4 * ng < valid) oa[j].x = y[0];
-              if (4 * ng + 1 < valid) oa[j].y = y[1];
-              if (4 * ng + 2 < valid) oa[j].z = y[2];
-            }
+            if (full4) oa[j] = *reinterpret_cast<const float4 *>(y);
           } else if (rope) {
             const size_t ti = (size_t)spos[t] * half + (cm & (half - 1));
             oa[j] = *reinterpret_cast<const float4 *>(p.cos_t + ti);
@@ -591,19 +587,12 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_tc_kernel(const __grid_consta
             float sq = 0.f;
 #pragma unroll
             for (int e = 0; e < 4; ++e)
-              if (4 * ng + e < valid) sq += yn[e] * yn[e];
+              if (full4) sq += yn[e] * yn[e];
             if (full4) {
               *reinterpret_cast<float4 *>(y) = make_float4(yn[0], yn[1], yn[2], yn[3]);
               __nv_bfloat162 lo = __floats2bfloat162_rn(gn[0] * yn[0], gn[1] * yn[1]);
               __nv_bfloat162 hi = __floats2bfloat162_rn(gn[2] * yn[2], gn[3] * yn[3]);
               *reinterpret_cast<uint2 *>(p.xb + (size_t)t * p.ldo + col) = make_uint2(*(uint32_t *)&lo, *(uint32_t *)&hi);
-            } else {
-#pragma unroll
-              for (int e = 0; e < 4; ++e)
-                if (4 * ng + e < valid) {
-                  y[e] = yn[e];
-                  p.xb[(size_t)t * p.ldo + col + e] = __float2bfloat16_rn(gn[e] * yn[e]);
-                }
             }
 #pragma unroll
             for (int o = 16; o; o >>= 1) sq += __shfl_xor_sync(0xffffffffu, sq, o);
@@ -632,10 +621,6 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_tc_kernel(const __grid_consta
             if (full4) {
               __nv_bfloat162 lo = __floats2bfloat162_rn(rv[0], rv[1]), hi = __floats2bfloat162_rn(rv[2], rv[3]);
               *reinterpret_cast<uint2 *>(dst) = make_uint2(*(uint32_t *)&lo, *(uint32_t *)&hi);
-            } else {
-#pragma unroll
-              for (int e = 0; e < 4; ++e)
-                if (4 * ng + e < valid) dst[e] = __float2bfloat16_rn(rv[e]);
             }
           }
           continue;
@@ -652,7 +637,7 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_tc_kernel(const __grid_consta
 #pragma unroll
             for (int e = 0; e < 4; ++e) {
               uint32_t uo = ordered_u32(vals[e]);
-              if (4 * ng + e < valid && uo > bu) { bu = uo; bi = col + e; }
+              if (full4 && uo > bu) { bu = uo; bi = col + e; }
             }
             const uint32_t mx = __reduce_max_sync(0xffffffffu, bu);
             const int src_lane = __ffs(__ballot_sync(0xffffffffu, bu == mx)) - 1;   // lowest lane = smallest index
@@ -665,14 +650,10 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_tc_kernel(const __grid_consta
           if (p.out_f32) {
             float *y = p.out_f32 + (size_t)t * p.ldo + col;
             const bool add = p.mode == MODE_RESIDUAL;
-            if (full4 && ((p.ldo & 3) == 0)) {
+            if (full4) {                                              // the row pitch is a multiple of 4 as well
               float4 o4 = make_float4(vals[0], vals[1], vals[2], vals[3]);
               if (add) { const float4 y4 = *reinterpret_cast<const float4 *>(y); o4.x += y4.x; o4.y += y4.y; o4.z += y4.z; o4.w += y4.w; }
               *reinterpret_cast<float4 *>(y) = o4;
-            } else {
-#pragma unroll
-              for (int e = 0; e < 4; ++e)
-                if (4 * ng + e < valid) y[e] = add ? y[e] + vals[e] : vals[e];
             }
           }
         }
