@@ -838,10 +838,9 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_tc_kernel(const __grid_consta
               p.tile_max[(size_t)s.tile * OURO_MAX_ROWS + t] = ordered_f32(bu);
               p.tile_arg[(size_t)s.tile * OURO_MAX_ROWS + t] = bi;
             }
-            if (p.out_f32) finish_plain(s.tile, et, 128, 0, 0, 1, 0, stage, c0, lim);
-          } else {
-            finish_plain(s.tile, et, 128, 0, 0, 1, 0, stage, c0, lim);
           }
+          // one call site for every other mode (the routine is inlined: a second site would be a second copy of it)
+          if (p.mode != MODE_SWIGLU && (p.mode != MODE_HEAD || p.out_f32)) finish_plain(s.tile, et, 128, 0, 0, 1, 0, stage, c0, lim);
           if (publish && c1 == p.t_pad) __threadfence();
           epi_barrier();
           if (publish && c1 == p.t_pad && et == 0) atomicAdd(cp.finished + ci, 1);
