@@ -205,6 +205,8 @@ __device__ __forceinline__ void mbox_post(int32_t *slot, const int32_t *payload,
 // Lookup with key d_gamma (warp 0) and packing in one launch.
 __global__ void lookup_assemble_kernel(PoolDev P, BlockDev b, DevState *st, const int32_t *draft, int32_t *suffix,
                                        int32_t *count, int L, int gamma, int S, int K) {
+  pdl_wait();            // launched while the kernel before it drains; it never lets its own successor start early (the
+                         // forward's kernels read the block description before their dependency wait)
   if (threadIdx.x < 32) {
     int32_t key = draft[gamma - 1];
     int n = (key < 0 || P.S == 0) ? 0 : pool_lookup(P, key, K, suffix);
@@ -237,7 +239,7 @@ void launch_assemble_candidates(const BlockDev &b, DevState *st, const int32_t *
 void launch_lookup_assemble(const PoolDev &P, const BlockDev &b, DevState *st, const int32_t *draft, int32_t *suffix,
                             int32_t *count, int L, int gamma, int S, int K, cudaStream_t s) {
   OURO_COUNT_LAUNCH();
-  lookup_assemble_kernel<<<1, OURO_MAX_ROWS, 0, s>>>(P, b, st, draft, suffix, count, L, gamma, S, K);
+  launch_pdl(lookup_assemble_kernel, 1, OURO_MAX_ROWS, 0, s, P, b, st, draft, suffix, count, L, gamma, S, K);
 }
 void launch_assemble_causal(const BlockDev &b, const int32_t *tokens, int n, int L, cudaStream_t s) {
   OURO_COUNT_LAUNCH();
@@ -346,6 +348,7 @@ __device__ void harvest_body(const BlockDev &b, DevState *st, const PoolDev &P, 
 __global__ void accept_compact_harvest_kernel(BlockDev b, DevState *st, PoolDev P, const int32_t *o, int32_t *seq_dev,
                                               unsigned char *k_cache, unsigned char *v_cache, int L, int gamma, int S,
                                               int max_seq, int row_bytes, unsigned flags, int32_t *mbox, int32_t seq) {
+  pdl_wait();            // its blocks are in place while the kernel that writes `o` finishes
   if (blockIdx.x == 0) {
     if (threadIdx.x == 0) {
       accept_body(b, st, o, seq_dev, gamma, S);
@@ -384,9 +387,8 @@ void launch_accept_compact_harvest(const BlockDev &b, DevState *st, const PoolDe
                                    unsigned flags, int32_t *mbox, int32_t seq, cudaStream_t s) {
   OURO_COUNT_LAUNCH();
   const int es = d.dtype == OURO_BF16 ? 2 : 4;
-  accept_compact_harvest_kernel<<<1 + S * d.n_layers * 2, 128, 0, s>>>(b, st, P, o, seq_dev, (unsigned char *)k_cache,
-                                                                      (unsigned char *)v_cache, L, gamma, S, d.max_seq,
-                                                                      d.n_kv_heads * d.head_dim * es, flags, mbox, seq);
+  launch_pdl(accept_compact_harvest_kernel, 1 + S * d.n_layers * 2, 128, 0, s, b, st, P, o, seq_dev, (unsigned char *)k_cache,
+             (unsigned char *)v_cache, L, gamma, S, (int)d.max_seq, d.n_kv_heads * d.head_dim * es, flags, mbox, seq);
 }
 
 // ------------------------------------------------------------- phrase-level drafting (Section 3.1)
