@@ -491,8 +491,9 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_tc_kernel(const __grid_consta
         wait_flag[4 + grp] = counter_wait(p.counters + tile, n, p.status, p.wait_limit) && !*abort_flag;
         TRACE(6);
       }
+      // The polling thread's acquire and the barrier order the others' reads of the partial sums behind the
+      // contributors' releases; those reads go to L2 (ld.global.cg), so no fence of their own is needed.
       if (G == 128) epi_barrier(); else group_barrier(grp);
-      __threadfence();
       if (gi == 0 && grp == 0) TRACE(9);
       return wait_flag[4 + grp] != 0;
     };
