@@ -352,14 +352,28 @@ __global__ void __launch_bounds__(THREADS, 1) attn_tm_kernel(const __grid_consta
   pdl_wait();
   if (tid == 0) TRACE(2);
   // ---- Q tile: K-major, two halves of 64 dims, 128-byte swizzle; rows without a query are zero
-  for (int idx = tid; idx < QR * 16; idx += THREADS) {
-    const int t = idx >> 4, ch = idx & 15, info = ms->map[t];
-    uint4 val = make_uint4(0, 0, 0, 0);
-    if (info >= 0) {
-      const int r = info & 0xff, hq = (info >> 8) & 0xff;
-      val = __ldg(reinterpret_cast<const uint4 *>(p.q + ((size_t)r * p.H + kvh * g + hq) * HD + ch * 8));
+  {
+    // every thread's pieces are requested before the first is stored: one round trip to L2 instead of one per piece
+    constexpr int QI = (QR * 16 + THREADS - 1) / THREADS;
+    uint4 val[QI];
+#pragma unroll
+    for (int i = 0; i < QI; ++i) {
+      const int idx = tid + i * THREADS, t = idx >> 4, ch = idx & 15;
+      val[i] = make_uint4(0, 0, 0, 0);
+      if (idx < QR * 16) {
+        const int info = ms->map[t];
+        if (info >= 0) {
+          const int r = info & 0xff, hq = (info >> 8) & 0xff;
+          val[i] = __ldg(reinterpret_cast<const uint4 *>(p.q + ((size_t)r * p.H + kvh * g + hq) * HD + ch * 8));
+        }
+      }
     }
-    *reinterpret_cast<uint4 *>(smem + OFF_Q + (ch >> 3) * HALF + t * 128 + (((ch & 7) ^ (t & 7)) << 4)) = val;
+#pragma unroll
+    for (int i = 0; i < QI; ++i) {
+      const int idx = tid + i * THREADS, t = idx >> 4, ch = idx & 15;
+      if (idx < QR * 16)
+        *reinterpret_cast<uint4 *>(smem + OFF_Q + (ch >> 3) * HALF + t * 128 + (((ch & 7) ^ (t & 7)) << 4)) = val[i];
+    }
   }
   fence_async_smem();
   fence_before_sync();
