@@ -52,6 +52,7 @@ using ws::TILE_N;
 using ws::Span;
 constexpr int A_BYTES = TILE_N * BLOCK_K * 2;
 constexpr int THREADS = 224;      // warp 0 weight TMA, warp 1 MMA, warps 2..5 epilogue, warp 6 activation TMA
+constexpr int W_PRODUCERS = 2;    // lanes of warp 0 that issue the weight copies, stage by stage in turn (a power of two, smaller than the ring)
 constexpr int MAX_GRID = 160;
 constexpr int SLOT_FLOATS = TILE_N * OURO_MAX_ROWS;
 constexpr uint32_t SPIN_LIMIT = 1u << 24;
@@ -298,7 +299,7 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_tc_kernel(const __grid_consta
 
   if (warp == 0) {
     // ---------------------------------------------------------------- TMA producer
-    if (lane == 0) {
+    if (lane < W_PRODUCERS) {
       // The weights do not depend on the previous kernel, so this warp never waits for it: the ring fills with
       // weight tiles while the predecessor drains.  The activation tiles come from warp 6, after its wait.
       // One thread runs this loop once per 16 KB stage; at 40 GB/s per SM that is every 0.4 us, so the loop carries
@@ -317,16 +318,18 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_tc_kernel(const __grid_consta
         const CUtensorMap *m0 = &p.a[seg];
         uint8_t *sa = ring + (size_t)st * stage_bytes;
         for (int kb = s.kb0; kb < s.kb1; ++kb, ++n) {
-          if (round > 0) {
-            ok = mbar_wait(&empty[st], (round - 1) & 1, abort_flag) && !*abort_flag;
-            if (!ok) break;
-          }
-          mbar_expect_tx(&full[st], A_BYTES);
-          if (swiglu) {
-            tma_load_2d(sa, &p.a[0], &full[st], kb * BLOCK_K, row0, HINT_EVICT_FIRST);
-            tma_load_2d(sa + A_BYTES / 2, &p.a[1], &full[st], kb * BLOCK_K, row0, HINT_EVICT_FIRST);
-          } else {
-            tma_load_2d(sa, m0, &full[st], kb * BLOCK_K, row0, HINT_EVICT_FIRST);
+          if ((n & (W_PRODUCERS - 1)) == (uint32_t)lane) {           // the lanes take the stages in turn
+            if (round > 0) {
+              ok = mbar_wait(&empty[st], (round - 1) & 1, abort_flag) && !*abort_flag;
+              if (!ok) break;
+            }
+            mbar_expect_tx(&full[st], A_BYTES);
+            if (swiglu) {
+              tma_load_2d(sa, &p.a[0], &full[st], kb * BLOCK_K, row0, HINT_EVICT_FIRST);
+              tma_load_2d(sa + A_BYTES / 2, &p.a[1], &full[st], kb * BLOCK_K, row0, HINT_EVICT_FIRST);
+            } else {
+              tma_load_2d(sa, m0, &full[st], kb * BLOCK_K, row0, HINT_EVICT_FIRST);
+            }
           }
           sa += stage_bytes;
           if (++st == n_stages) { st = 0; ++round; sa = ring; }
@@ -877,7 +880,7 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_tc_kernel(const __grid_consta
   // ------------------------------------------------------------------ teardown
   fence_before_sync();
   __syncthreads();
-  if (*abort_flag && lane == 0 && (warp == 0 || warp == 6)) {
+  if (*abort_flag && ((warp == 0 && lane < W_PRODUCERS) || (warp == 6 && lane == 0))) {
     // Somebody gave up: copies this lane issued may still be landing in this CTA's shared memory.  Wait (bounded) for
     // the last one of every stage before the CTA leaves; a stage whose other half was never requested cannot
     // complete its phase, which the limit covers (the bytes themselves arrive within microseconds).
