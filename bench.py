@@ -439,8 +439,8 @@ def run_generate(args, device):
 
 
 def generation_summary(device, tokens):
-    """BASELINE's other half: generated tokens/s at batch 1 on the 7B-shaped target with the 1.1B-shaped draft model
-    (configs[2]), plain greedy decoding against Ouroboros with replayed drafts (middle agreement level) without and
+    """The metric's other half: generated tokens/s at batch 1 on the 7B-shaped target with the 1.1B-shaped draft model
+    (configuration C3), plain greedy decoding against Ouroboros with replayed drafts (middle agreement level) without and
     with the replayed phrase source.  A short run: `tokens` generated tokens per mode."""
     import dataclasses
     from paper_2402_13720_b200 import binding
