@@ -84,6 +84,35 @@ __device__ void pool_erase(const PoolDev &P, const int32_t *phrase) {
 __device__ int pool_lookup(const PoolDev &P, int32_t key, int K, int32_t *suffix_out) {
   int lane = threadIdx.x & 31;
   int set = pool_set(P, key);
+  if (P.ways <= 32) {
+    // One way per lane: key and stamp are read once, the K newest are picked with shuffles alone, and all their
+    // suffixes are fetched together: two round trips to memory whatever K is.  (Stamps start at 1 and are unique.)
+    u64 mine = 0;
+    if (lane < P.ways) {
+      const int e = set * P.ways + lane;
+      if (P.key[e] == key) mine = P.stamp[e];
+    }
+    int found = 0, sel = -1;                       // lane f remembers the way of the f-th newest phrase
+    for (; found < K; ++found) {
+      u64 best = mine;
+      int best_w = mine ? lane : -1;
+#pragma unroll
+      for (int o = 16; o; o >>= 1) {
+        u64 s2 = __shfl_xor_sync(FULL, best, o);
+        int w2 = __shfl_xor_sync(FULL, best_w, o);
+        if (s2 > best) { best = s2; best_w = w2; }
+      }
+      if (best_w < 0) break;
+      if (lane == best_w) mine = 0;
+      if (lane == found) sel = best_w;
+    }
+    for (int idx0 = 0; idx0 < found * P.S; idx0 += 32) {
+      const int idx = idx0 + lane, f = min(idx / P.S, found - 1);
+      const int w = __shfl_sync(FULL, sel, f);
+      if (idx < found * P.S) suffix_out[idx] = P.suf[(size_t)(set * P.ways + w) * P.S + (idx - f * P.S)];
+    }
+    return found;
+  }
   u64 bound = ~0ull;
   int found = 0;
   for (; found < K; ++found) {
