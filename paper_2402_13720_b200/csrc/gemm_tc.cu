@@ -97,8 +97,9 @@ struct GemmParams {
   int ss_tiles;
   float ss_inv_d, eps;
   float *scratch;     // [grid][2][t][128] partial tiles
-  int *counters;      // [tiles] partial tiles published, zero between launches
-  int *done;          // [tiles] contributors that finished their share, zero between launches
+  int *counters;      // [tiles] partial tiles published, as (gen << 8) + count: a word left by an earlier GEMM is
+                      // smaller than this GEMM's (gen << 8), so nothing has to be cleared between GEMMs or launches
+  int gen;            // this GEMM's generation number (1 .. 2^22, grows with every GEMM the context runs)
   int *status;        // context status word
   int trace_id;           // which GEMM of the layer this is (timeline builds only)
   uint32_t wait_limit;    // polls of a partial-tile wait before it gives up (1 << 22 unless a test shortens it)
@@ -491,7 +492,7 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_tc_kernel(const __grid_consta
     // Returns false when the wait gave up.
     auto others_there = [&](int tile, int n, int gi, int grp, int G) -> bool {
       if (gi == 0) {
-        wait_flag[4 + grp] = counter_wait(p.counters + tile, n, p.status, p.wait_limit) && !*abort_flag;
+        wait_flag[4 + grp] = counter_wait(p.counters + tile, (p.gen << 8) + n, p.status, p.wait_limit) && !*abort_flag;
         TRACE(6);
       }
       // The polling thread's acquire and the barrier order the others' reads of the partial sums behind the
@@ -740,14 +741,9 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_tc_kernel(const __grid_consta
         if (mine) {
           if (publish) __threadfence();                                // this thread's outputs, before the tile counts as finished
           group_barrier(grp);
-          if (gi == 0) {                                               // the last contributor to finish re-arms the tile
-            int d = atomicAdd(p.done + tile, 1);
-            if (d == n - 1) {
-              p.counters[tile] = 0;
-              p.done[tile] = 0;
-              if (publish) { __threadfence(); atomicAdd(cp.finished + ci, 1); }
-            }
-          }
+          // every contributor counts towards the hand-over itself: the GEMM is finished once all shares of all tiles
+          // are (the host passes the total), and nobody has to learn that it was the last of its tile
+          if (gi == 0 && publish) atomicAdd(cp.finished + ci, 1);
         }
       }
       if (gi == 0 && grp == 0) TRACE(11);
@@ -863,7 +859,10 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_tc_kernel(const __grid_consta
         if (lane == 0) mbar_arrive(&acc_empty[a]);
         __threadfence();
         epi_barrier();
-        if (et == 0) atomicAdd(p.counters + s.tile, 1);
+        if (et == 0) {                             // first of this generation to get here: replaces what an earlier GEMM left
+          atomicMax(p.counters + s.tile, p.gen << 8);
+          atomicAdd(p.counters + s.tile, 1);
+        }
         pend_tile[n_pend] = s.tile;
         pend_n[n_pend] = s.n_contrib;
         pend_first[n_pend] = s.first_owner;
@@ -944,6 +943,7 @@ struct FastState {
   int chain_kind[MAX_CHAIN] = {0, 0, 0, 0};
   bool fuse = true;             // run consecutive GEMMs as one launch
   long pf_ffn_rows = 0;         // rows of gate and of up the attention kernel prefetches into L2 besides the output projection (< 0: nothing)
+  int gen_next = 1;             // generation number of the next GEMM (tile counters carry it, see GemmParams::counters)
   bool dirty = false;           // a bounded wait gave up: counters must be cleared before the next launch
   uint32_t wait_limit = 1u << 22;   // polls of a partial-tile wait (ouro_debug_set_wait_limit)
 };
@@ -1116,6 +1116,16 @@ static int grid_for(const FastState &s, int tiles, int kb) {
   const long total = (long)tiles * kb;
   return total < s.grid ? (int)total : s.grid;
 }
+// What the hand-over counter of a GEMM reaches: one count per whole tile and one per contributor of a split tile
+// (the schedule of weight_stream.cuh, worked out on the host).
+static int finish_units(int tiles, int kb, int grid) {
+  const int t0 = (tiles / grid) * grid, rem = tiles - t0;
+  if (rem == 0) return tiles;
+  const int total = rem * kb, per = (total + grid - 1) / grid;
+  int units = t0;
+  for (int rel = 0; rel < rem; ++rel) units += (rel * kb + kb - 1) / per - (rel * kb) / per + 1;
+  return units;
+}
 // Launches the GEMMs collected so far as one chain.
 static void flush_chain(ouro_ctx *c) {
   FastState &s = c->fast->s;
@@ -1125,7 +1135,12 @@ static void flush_chain(ouro_ctx *c) {
   int grid = 1;
   for (int i = 0; i < cp.n; ++i) grid = std::max(grid, grid_for(s, cp.g[i].tiles, cp.g[i].kb));
   cp.finished = s.finished;
-  for (int i = 0; i + 1 < cp.n; ++i) cp.target[i] = (s.finished_host[i] += cp.g[i].tiles);
+  if (s.gen_next + MAX_CHAIN >= (1 << 22)) {                 // generation numbers used up: start over on cleared words
+    cudaMemsetAsync(s.counters, 0, MAX_TILES * sizeof(int), c->stream);
+    s.gen_next = 1;
+  }
+  for (int i = 0; i < cp.n; ++i) cp.g[i].gen = s.gen_next++;
+  for (int i = 0; i + 1 < cp.n; ++i) cp.target[i] = (s.finished_host[i] += finish_units(cp.g[i].tiles, cp.g[i].kb, grid));
   if (cp.fold.part || cp.embed.table) cp.fold_target = (s.finished_host[MAX_CHAIN] += grid);
   const bool per_kind = cp.n == 1 && c->prof_class >= OURO_PROF_QKV && c->prof_class <= OURO_PROF_HEAD;
   static const int kind_class[5] = {OURO_PROF_QKV, OURO_PROF_WO, OURO_PROF_GATEUP, OURO_PROF_DOWN, OURO_PROF_HEAD};
@@ -1148,7 +1163,6 @@ static void push_gemm(ouro_ctx *c, GemmParams &p, int kind, const CUtensorMap *x
   p.stages = stages_for(p.t_pad, s.smem_max);
   p.scratch = s.slots;
   p.counters = s.counters;
-  p.done = s.counters + MAX_TILES;
   p.status = &c->st->status;
   p.rows_dev = c->cur_rows_dev;
   p.trace_id = kind;
@@ -1171,6 +1185,7 @@ void ouro_fast_reset(ouro_ctx *c, bool force) {
   if (!force && !s.dirty) return;
   cudaMemsetAsync(s.counters, 0, 2 * MAX_TILES * sizeof(int) + SPARE_BYTES, c->stream);
   for (int &v : s.finished_host) v = 0;
+  s.gen_next = 1;
   s.dirty = false;
 }
 void ouro_fast_mark_dirty(ouro_ctx *c) {
@@ -1488,7 +1503,7 @@ extern "C" int ouro_lm_head_static(const void *x_dev, const void *lm_head_dev, i
   p.wait_limit = 1u << 22;
   p.scratch = (float *)base;
   p.counters = (int *)(base + NA_OFF_COUNTERS);
-  p.done = p.counters + NA_MAX_TILES;
+  p.gen = 1;                                   // the words were cleared just above
   p.status = (int *)(base + NA_OFF_STATUS);
   const int total = tiles * p.kb;
   gemm_tc_kernel<<<total < NA_GRID ? total : NA_GRID, THREADS, g_na_smem[dev], s>>>(cp);
