@@ -1009,6 +1009,8 @@ int ouro_fast_setup(ouro_ctx *c) {
     f->s.fuse = !(e && e[0] == '0');
     const char *pf = getenv("OURO_PF_ROWS");
     if (pf) f->s.pf_ffn_rows = atol(pf);
+    const char *g0 = getenv("OURO_GEN_START");                  // test aid: first generation number of the tile counters
+    if (g0 && atoi(g0) > 0 && atoi(g0) < (1 << 22)) f->s.gen_next = atoi(g0);
   }
   f->s.tile_max = (float *)((char *)c->a.scratch + slots_bytes() + 2 * MAX_TILES * sizeof(int) + SPARE_BYTES);
   f->s.tile_arg = (int *)((char *)f->s.tile_max + tile_best_bytes());

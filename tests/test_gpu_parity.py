@@ -852,6 +852,27 @@ def test_bounded_wait_gives_up_and_the_context_recovers():
     eng.close()
 
 
+def test_tile_counter_generations_wrap_around(monkeypatch):
+    """The split-K tile counters carry a generation number that grows with every GEMM; when the numbers are used up
+    the words are cleared and counting starts over.  Started a few hundred GEMMs before that point, a generation
+    crosses it and must still equal plain decoding token for token (which crosses it at another place)."""
+    monkeypatch.setenv("OURO_GEN_START", str((1 << 22) - 300))
+    P = synth.DecodeParams(4, 9, 4, 32, 8)
+    eng, _ = make(MIDB, P, 5)
+    prompt = synth.prompt(5, MIDB.vocab, 64, 0.3, 8, 32)
+    van, _ = eng.generate_vanilla(prompt, 48)
+    truth = np.concatenate([prompt, van, np.zeros(32, dtype=np.int32)])
+    eng.set_drafter(lambda seq, g, step: synth.corrupt_drafts(1, truth, len(seq), g, MIDB.vocab, 0.1, 0.05, step))
+    out, stats = eng.generate(prompt, 48)
+    eng.set_drafter(None)
+    assert np.array_equal(out, van) and stats["target_calls"] < 48
+    eng.close()
+    monkeypatch.delenv("OURO_GEN_START")
+    eng2, _ = make(MIDB, P, 5)                       # and the same text from the usual starting point
+    assert np.array_equal(eng2.generate_vanilla(prompt, 48)[0], van)
+    eng2.close()
+
+
 # ------------------------------------------------- phrase generation during the draft forward (Section 3.1)
 
 def test_lookahead_window_matches_oracle_c1():
