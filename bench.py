@@ -328,21 +328,36 @@ def run_generate(args, device):
         "window": Pw.window, "tokens_per_s": len(out) / (st["ms_total"] * 1e-3), "target_calls": st["target_calls"],
         "candidates": st["candidates"], "suffix_tokens": st["suffix_tokens"],
         "ms_draft_per_step": st["ms_draft"] / st["target_calls"], "identical_to_vanilla": bool(np.array_equal(out, van))}
-    # History reuse (Section 3.4): the same query again with the pool of the first run, and another query with it.
-    cold, stc = eng3.generate(prompt, gen)
-    warm, stw = eng3.generate(prompt, gen, keep_pool=True)
+    # History reuse (Section 3.4): the pool of earlier queries is kept for the next one.  Replayed drafts at the middle
+    # agreement level, nothing injected from the host: the phrases come from the accepted text of the earlier run
+    # (extension OURO_HARVEST_ACCEPTED) and from the verification's own corrections.  The same query again finds its
+    # own continuation in the pool; another query finds little (synthetic texts share no phrases), which is the case
+    # the paper's Table on context locality contrasts.
+    mid = lambda truth_: (lambda seq, g, step: synth.corrupt_drafts(SEED + 7, truth_, len(seq), g, T.vocab, 0.12, 0.03, step))
     other = synth.prompt(SEED + 1, T.vocab, R["n"], R["copy_frac"], *R["span"])
-    o_cold, sto_c = eng3.generate(other, gen)
-    eng3.generate(prompt, gen)
-    o_warm, sto_w = eng3.generate(other, gen, keep_pool=True)
+    van_o, _ = eng.generate_vanilla(other, gen)
+    truth_o = np.concatenate([other, van_o, np.zeros(64, dtype=np.int32)])
+    eng.set_drafter(mid(truth))
+    cold, stc = eng.generate(prompt, gen)
+    warm, stw = eng.generate(prompt, gen, keep_pool=True)
+    eng.set_drafter(mid(truth_o))
+    o_cold, sto_c = eng.generate(other, gen)
+    eng.set_drafter(mid(truth))
+    eng.generate(prompt, gen)
+    eng.set_drafter(mid(truth_o))
+    o_warm, sto_w = eng.generate(other, gen, keep_pool=True)
+    eng.set_drafter(None)
     tps = lambda o, st_: round(len(o) / (st_["ms_total"] * 1e-3), 1)
     res["history_reuse"] = {
+        "drafts": "replay_mid",
         "same_query": {"cold_tokens_per_s": tps(cold, stc), "warm_tokens_per_s": tps(warm, stw),
                        "cold_target_calls": stc["target_calls"], "warm_target_calls": stw["target_calls"],
-                       "warm_suffix_tokens": stw["suffix_tokens"], "identical": bool(np.array_equal(cold, warm))},
+                       "cold_suffix_tokens": stc["suffix_tokens"], "warm_suffix_tokens": stw["suffix_tokens"],
+                       "identical": bool(np.array_equal(cold, warm) and np.array_equal(cold, van))},
         "other_query": {"cold_tokens_per_s": tps(o_cold, sto_c), "warm_tokens_per_s": tps(o_warm, sto_w),
                         "cold_target_calls": sto_c["target_calls"], "warm_target_calls": sto_w["target_calls"],
-                        "identical": bool(np.array_equal(o_cold, o_warm))}}
+                        "warm_suffix_tokens": sto_w["suffix_tokens"],
+                        "identical": bool(np.array_equal(o_cold, o_warm) and np.array_equal(o_cold, van_o))}}
     eng3.close()
 
     # Algorithm 1 of the paper's Appendix B: coordinate search of gamma, W and beta on the wall-clock time of this
