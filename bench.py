@@ -455,8 +455,8 @@ def run_generate(args, device):
 
 def generation_summary(device, tokens):
     """The metric's other half: generated tokens/s at batch 1 on the 7B-shaped target with the 1.1B-shaped draft model
-    (configuration C3), plain greedy decoding against Ouroboros with replayed drafts (middle agreement level) without and
-    with the replayed phrase source.  A short run: `tokens` generated tokens per mode."""
+    (configuration C3), plain greedy decoding against Ouroboros with replayed drafts (middle agreement level), the same
+    with the pool of the run before (history reuse), and with the replayed phrase source.  A short run: `tokens` generated tokens per mode."""
     import dataclasses
     from paper_2402_13720_b200 import binding
     T, D, P, R = synth.config("C3")
@@ -471,9 +471,9 @@ def generation_summary(device, tokens):
                      f"beta {P.beta}, K {P.K}",
            "vanilla": {"tokens_per_s": round(len(van) / (vs["ms_total"] * 1e-3), 1)}}
 
-    def run(name, drafter):
+    def run(name, drafter, keep_pool=False):
         eng.set_drafter(drafter)
-        o, st = eng.generate(prompt, tokens)
+        o, st = eng.generate(prompt, tokens, keep_pool=keep_pool)
         eng.set_drafter(None)
         out[name] = {"tokens_per_s": round(len(o) / (st["ms_total"] * 1e-3), 1),
                      "vs_vanilla": round(len(o) / (st["ms_total"] * 1e-3) / out["vanilla"]["tokens_per_s"], 3),
@@ -495,6 +495,8 @@ def generation_summary(device, tokens):
         return d
 
     run("replayed_drafts", drafts)
+    # Section 3.4, history reuse: the same query once more with the pool the run above left behind (nothing injected)
+    run("replayed_drafts_warm_pool", drafts, keep_pool=True)
     run("replayed_drafts_and_phrases", drafts_and_phrases)
     eng.close()
     return out
